@@ -1,0 +1,533 @@
+"""Pins for the CPU oracle: each part is checked against something other than itself
+(published known-answer vectors, closed forms, invariants, library routines, a worked
+example, brute force on tiny inputs)."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import OracleState
+
+
+def read_golden(path):
+    out = {}
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        k, *vals = line.split()
+        out[k] = np.array([float(v) for v in vals], np.float64)
+    return out
+
+
+# ---------------------------------------------------------------- S1: Philox, z
+def test_philox_known_answers(orc, golden_dir):
+    n = 0
+    for line in open(os.path.join(golden_dir, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(v, 16) for v in line.split()]
+        assert orc.philox(w[0:4], w[4:6]) == w[6:10]
+        n += 1
+    assert n == 3
+
+
+def test_philox_is_bijection_on_small_sample(orc):
+    # distinct counters under one key give distinct outputs (a keyed bijection)
+    seen = set()
+    for c0 in range(64):
+        for c1 in range(4):
+            seen.add(tuple(orc.philox([c0, c1, 7, 0], [123, 456])))
+    assert len(seen) == 256
+
+
+def test_z_definition_matches_row_generator(orc):
+    # per-element definition (one Philox call per element) vs the per-128 cached rows
+    K, P = 3, 1000
+    z = orc.sample_z(0x5EED0001, 17, K, P)
+    bits = orc.sample_zbits(0x5EED0001, 17, K, P)
+    assert np.array_equal(z, np.where(bits == 1, -1.0, 1.0).astype(np.float32))
+    assert set(np.unique(z)) == {-1.0, 1.0}
+
+
+def test_z_bit_layout_by_hand(orc):
+    # element j uses bit (j & 31) of word (j >> 5) & 3 of block j >> 7
+    seed, t, i = 0x0123456789ABCDEF, 5, 2
+    bits = orc.sample_zbits(seed, t, i + 1, 300)[i]
+    for j in (0, 1, 31, 32, 95, 127, 128, 200, 299):
+        r = orc.philox([j >> 7, i, t, 0], [seed & 0xffffffff, seed >> 32])
+        assert bits[j] == (r[(j >> 5) & 3] >> (j & 31)) & 1
+
+
+def test_z_counter_uniqueness(orc):
+    base = orc.sample_zbits(1, 1, 2, 256)
+    assert not np.array_equal(base, orc.sample_zbits(2, 1, 2, 256))          # seed
+    assert not np.array_equal(base, orc.sample_zbits(1, 2, 2, 256))          # round
+    assert not np.array_equal(base[0], base[1])                               # worker
+    assert not np.array_equal(base[0, :128], base[0, 128:])                   # block
+    assert not np.array_equal(base, orc.sample_zbits(1 << 32 | 1, 1, 2, 256))  # high key word
+
+
+def test_z_statistics(orc):
+    K, P = 4, 1 << 18
+    z = orc.sample_z(99, 3, K, P).astype(np.float64)
+    n = K * P
+    assert abs(z.mean()) < 5 / math.sqrt(n)
+    assert abs((z[:, 1:] * z[:, :-1]).mean()) < 5 / math.sqrt(n)          # lag 1
+    assert abs((z[0] * z[1]).mean()) < 5 / math.sqrt(P)                   # across workers
+    z2 = orc.sample_z(99, 4, K, P).astype(np.float64)
+    assert abs((z * z2).mean()) < 5 / math.sqrt(n)                        # across rounds
+
+
+# ------------------------------------------------------ a2/a3: Hutchinson, averaging
+def test_hutchinson_exact_on_diagonal_quadratic(orc):
+    # H = diag(h): z (.) (H z) = h exactly for any Rademacher z (Sec. IV-B); then the
+    # second moment after one step is (1-beta2) h^2 and x moves by lr*g/(h+eps).
+    P, K = 777, 2
+    rng = np.random.default_rng(0)
+    h = rng.uniform(0.1, 10, P).astype(np.float32)
+    x0 = rng.standard_normal(P).astype(np.float32)
+    st = OracleState(x0, K, [(0, P, 1)])
+    z = orc.sample_z(5, 1, K, P)
+    hvp = (h[None] * z).astype(np.float32)
+    g = (h[None] * st.x).astype(np.float32)
+    st.local_step(g, hvp, 5, 1, lr=0.1)
+    omb2 = np.float32(1) - np.float32(0.999)
+    assert np.array_equal(st.v, np.broadcast_to((omb2 * h) * h, (K, P)))
+    # closed form of the first step: x1 = x0 - lr * g / (|h| + eps), in double
+    x1 = x0.astype(np.float64) - 0.1 * g[0].astype(np.float64) / (h.astype(np.float64) + 1e-4)
+    assert np.allclose(st.x[0], x1, rtol=2e-6, atol=1e-7)
+
+
+def test_hutchinson_dense_tiny_converges_to_diagonal(orc):
+    # dense symmetric H (P=6): the mean over rounds of z (.) (H z) tends to diag(H)
+    P, T = 6, 4000
+    rng = np.random.default_rng(1)
+    A = rng.standard_normal((P, P))
+    H = A @ A.T
+    acc = np.zeros(P)
+    for t in range(1, T + 1):
+        z = orc.sample_z(11, t, 1, P)[0].astype(np.float64)
+        acc += z * (H @ z)
+    off = np.sqrt(((H - np.diag(np.diag(H))) ** 2).sum(1))
+    assert np.all(np.abs(acc / T - np.diag(H)) < 5 * off / math.sqrt(T))
+
+
+def test_spatial_average_properties(orc):
+    rng = np.random.default_rng(2)
+    segs = [(0, 18, 9), (18, 7, 1), (25, 98, 49), (130, 8, 4)]   # gap 123..129
+    P = 140
+    d = rng.standard_normal(P).astype(np.float32)
+    out = orc.spatial_average(d, segs)
+    # identity where block = 1, in gaps, and after the last segment
+    assert np.array_equal(out[18:25], d[18:25])
+    assert np.array_equal(out[123:130], d[123:130])
+    assert np.array_equal(out[138:], d[138:])
+    # constant inside a block, equal to the mean; block sums preserved
+    for off, n, b in segs:
+        if b == 1:
+            continue
+        for q in range(off, off + n, b):
+            blk = out[q:q + b]
+            assert np.all(blk == blk[0])
+            assert abs(float(blk[0]) - d[q:q + b].astype(np.float64).mean()) < 1e-6
+    # idempotent up to the rounding of summing b equal values (b <= 49 here)
+    again = orc.spatial_average(out, segs)
+    assert np.allclose(again, out, rtol=4e-6, atol=0)
+    # worked example: (2,-1 | 3,1) with block 2 -> (0.5,0.5 | 2,2)
+    ex = orc.spatial_average(np.array([2, -1, 3, 1], np.float32), [(0, 4, 2)])
+    assert np.array_equal(ex, np.array([0.5, 0.5, 2, 2], np.float32))
+
+
+def test_spatial_average_order_is_ascending(orc):
+    # ((1e8 + 1) + -1e8) in binary32 is 0, not 1: pins the left-to-right order
+    ex = orc.spatial_average(np.array([1e8, 1.0, -1e8], np.float32), [(0, 3, 3)])
+    assert np.array_equal(ex, np.zeros(3, np.float32))
+    ex = orc.spatial_average(np.array([1e8, -1e8, 1.0], np.float32), [(0, 3, 3)])
+    assert np.allclose(ex, np.float32(1.0) / np.float32(3.0), rtol=0, atol=0)
+
+
+# ----------------------------------------------------- a4/a5: moments and update
+def test_step_reduces_to_adam(orc):
+    # With hvp := z (.) g and block 1 the Hutchinson diagonal equals g, so the step is
+    # Adam (Sec. IV-B: "similar to ADAM ... gradient replaced by the ... Hessian diagonal").
+    torch = pytest.importorskip("torch")
+    P, K, T = 513, 1, 25
+    rng = np.random.default_rng(3)
+    x0 = rng.standard_normal(P).astype(np.float32)
+    st = OracleState(x0, K, [(0, P, 1)])
+    p = torch.tensor(x0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.Adam([p], lr=0.01, betas=(float(np.float32(0.9)), float(np.float32(0.999))),
+                           eps=1e-4)
+    for t in range(1, T + 1):
+        g = rng.standard_normal((K, P)).astype(np.float32)
+        z = orc.sample_z(42, t, K, P)
+        st.local_step(g, (z * g).astype(np.float32), 42, t, lr=0.01, eps=1e-4)
+        p.grad = torch.tensor(g[0].astype(np.float64))
+        opt.step()
+    assert np.allclose(st.x[0], p.detach().numpy(), rtol=1e-5, atol=1e-6)
+
+
+def test_noise_free_quadratic_recurrence(orc):
+    # On f = 1/2 sum h x^2 without noise, vhat = h^2 at every step, so
+    # x_{t+1} = x_t - lr * mhat_t / (h + eps): a scalar linear recurrence (double).
+    P, T, lr, eps = 64, 40, 0.1, 1e-4
+    rng = np.random.default_rng(4)
+    h = rng.uniform(0.1, 10, P).astype(np.float32)
+    x0 = rng.standard_normal(P).astype(np.float32)
+    st = OracleState(x0, 1, [(0, P, 1)])
+    b1 = float(np.float32(0.9))
+    xd, md, hd = x0.astype(np.float64), np.zeros(P), h.astype(np.float64)
+    for t in range(1, T + 1):
+        z = orc.sample_z(1, t, 1, P)
+        g = (h[None] * st.x).astype(np.float32)
+        st.local_step(g, (h[None] * z).astype(np.float32), 1, t, lr=lr, eps=eps)
+        md = b1 * md + (1 - b1) * (hd * xd)
+        xd = xd - lr * (md / (1 - b1 ** t)) / (hd + eps)
+    assert np.allclose(st.x[0], xd, rtol=2e-5, atol=2e-6)
+
+
+def test_hessian_power_and_weight_decay_first_step(orc):
+    # step 1: mhat = g, vhat = dbar^2 -> x1 = x0 - lr*(g/(|dbar|^k + eps) + wd*x0)
+    P = 32
+    rng = np.random.default_rng(5)
+    x0 = rng.standard_normal(P).astype(np.float32)
+    g = rng.standard_normal((1, P)).astype(np.float32)
+    hv = rng.standard_normal((1, P)).astype(np.float32)
+    for k in (1.0, 0.5, 0.75):
+        st = OracleState(x0, 1, [(0, P, 1)])
+        st.local_step(g, hv, 9, 1, lr=0.05, eps=1e-3, hessian_power=k, weight_decay=0.01)
+        want = x0 - 0.05 * (g[0].astype(np.float64) / (np.abs(hv[0].astype(np.float64)) ** k + 1e-3)
+                            + 0.01 * x0)
+        assert np.allclose(st.x[0], want, rtol=1e-5, atol=1e-6), k
+
+
+def test_inactive_worker_untouched(orc):
+    P, K = 40, 3
+    rng = np.random.default_rng(6)
+    st = OracleState(rng.standard_normal(P).astype(np.float32), K, [(0, P, 1)])
+    g = rng.standard_normal((K, P)).astype(np.float32)
+    st.local_step(g, g.copy(), 1, 1, lr=0.1)
+    before = (st.x.copy(), st.m.copy(), st.v.copy(), st.step.copy())
+    st.local_step(g, g.copy(), 1, 2, lr=0.1, active=np.array([1, 0, 1], np.uint8))
+    assert np.array_equal(st.x[1], before[0][1]) and np.array_equal(st.m[1], before[1][1])
+    assert np.array_equal(st.v[1], before[2][1]) and st.step[1] == 1
+    assert st.step[0] == 2 and not np.array_equal(st.x[0], before[0][0])
+
+
+# --------------------------------------------------------------- S3: distance
+def test_norm2_pairwise_tree_brute_force(orc):
+    # P=5 padded to 8: ((d0+d1)+(d2+d3)) + ((d4+0)+(0+0)), squares in double
+    x = np.array([[1.5, -2.25, 3.0, 0.1, 7.0]], np.float32)
+    c = np.array([0.5, 0.25, -1.0, 0.3, 6.5], np.float32)
+    d = [float(np.float32(a) - np.float32(b)) for a, b in zip(x[0], c)]
+    s = [v * v for v in d]
+    want = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + 0.0) + (0.0 + 0.0))
+    assert orc.norm2(x, c)[0] == want
+
+
+def test_norm2_against_exact_sum_and_tiles(orc):
+    rng = np.random.default_rng(7)
+    K, P = 2, 5000
+    x = rng.standard_normal((K, P)).astype(np.float32)
+    c = rng.standard_normal(P).astype(np.float32)
+    n2 = orc.norm2(x, c)
+    for i in range(K):
+        d = (x[i] - c).astype(np.float64)
+        exact = math.fsum(d * d)
+        assert abs(n2[i] - exact) <= 1e-13 * exact
+    # any aligned power-of-two tile is a subtree: summing tile results pairwise
+    # reproduces the whole (P = 4096 here so the tiles are exact subtrees)
+    P2, T = 4096, 512
+    tiles = [orc.norm2(x[:1, s:s + T].copy(), c[s:s + T].copy())[0] for s in range(0, P2, T)]
+    while len(tiles) > 1:
+        tiles = [tiles[k] + tiles[k + 1] for k in range(0, len(tiles), 2)]
+    assert tiles[0] == orc.norm2(x[:1, :P2].copy(), c[:P2].copy())[0]
+
+
+# ------------------------------------------------------------ S6: elastic exchange
+def _rand_state(K, P, seed):
+    rng = np.random.default_rng(seed)
+    st = OracleState(rng.standard_normal(P).astype(np.float32), K, [(0, P, 1)])
+    st.x += rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+    return st
+
+
+def test_exchange_alpha_zero_and_all_masked_are_identity(orc):
+    st = _rand_state(3, 50, 8)
+    x0, c0 = st.x.copy(), st.center.copy()
+    st.exchange(alpha=0.0)
+    assert np.array_equal(st.x, x0) and np.array_equal(st.center, c0)
+    st.exchange(mask=np.zeros(3, np.uint8), alpha=0.3)
+    assert np.array_equal(st.x, x0) and np.array_equal(st.center, c0)
+
+
+def test_exchange_reduces_to_easgd(orc):
+    # h1 = h2 = alpha, nobody down: the synchronous EASGD update (Eqs. 8-9 oriented as
+    # Eqs. 12-13): x_i' = x_i - alpha (x_i - c), c' = (1 - K alpha) c + alpha sum_i x_i
+    K, P, al = 4, 64, 0.1
+    st = _rand_state(K, P, 9)
+    x0, c0 = st.x.astype(np.float64), st.center.astype(np.float64)
+    st.exchange(alpha=al)
+    a = float(np.float32(al))
+    assert np.allclose(st.center, (1 - K * a) * c0 + a * x0.sum(0), rtol=1e-6, atol=1e-6)
+    assert np.allclose(st.x, x0 - a * (x0 - c0), rtol=1e-6, atol=1e-6)
+    # equal coefficients conserve center + sum_i x_i
+    assert np.allclose(st.center.astype(np.float64) + st.x.astype(np.float64).sum(0),
+                       c0 + x0.sum(0), rtol=1e-6, atol=1e-6)
+
+
+def test_exchange_moves_worker_and_master_toward_each_other(orc):
+    # one worker: both distances to the old midpoint shrink (orientation of the pull)
+    st = OracleState(np.zeros(1, np.float32), 1, [(0, 1, 1)])
+    st.x[0, 0] = 1.0
+    st.exchange(alpha=0.25)
+    assert st.x[0, 0] == np.float32(0.75) and st.center[0] == np.float32(0.25)
+
+
+def test_exchange_failed_worker_weights(orc):
+    # h1 = 1, h2 = 0 for worker 1 (a < threshold): it is reset to the old master and
+    # contributes nothing to the new master (Sec. IV-A, last paragraph)
+    K, P = 3, 20
+    st = _rand_state(K, P, 10)
+    c0, x0 = st.center.copy(), st.x.copy()
+    h2 = np.array([0.1, 0.0, 0.1], np.float32)
+    h1 = np.array([0.1, 1.0, 0.1], np.float32)
+    st.exchange(h2=h2, h1=h1)
+    assert np.allclose(st.x[1], c0, atol=1e-7)
+    st2 = _rand_state(K, P, 10)
+    st2.exchange(mask=np.array([1, 0, 1], np.uint8), alpha=0.1)
+    assert np.array_equal(st.center, st2.center)          # master ignores worker 1
+    assert np.array_equal(st2.x[1], x0[1])                 # a masked worker is untouched
+
+
+def test_exchange_simultaneous_uses_old_center(orc):
+    # two workers at +1 and -1 around c = 0 cancel exactly in the master
+    st = OracleState(np.zeros(4, np.float32), 2, [(0, 4, 1)])
+    st.x[0] = 1.0
+    st.x[1] = -1.0
+    st.exchange(alpha=0.3)
+    assert np.array_equal(st.center, np.zeros(4, np.float32))
+    assert np.allclose(st.x[0], 0.7) and np.allclose(st.x[1], -0.7)
+
+
+# ------------------------------------------------------------------ S4: weights
+def test_h1_h2_closed_forms(orc):
+    al, ka = 0.1, -0.1
+    assert orc.h1(ka, al, ka) == 1.0 and orc.h2(ka, al, ka) == 0.0      # continuity at threshold
+    assert abs(orc.h1(0.0, al, ka) - al) < 1e-15 and orc.h2(0.0, al, ka) == al
+    assert orc.h1(1e-9, al, ka) == al and orc.h2(1e-9, al, ka) == al
+    assert orc.h1(-5.0, al, ka) == 1.0 and orc.h2(-5.0, al, ka) == 0.0
+    grid = np.linspace(-0.3, 0.3, 601)
+    v1 = np.array([orc.h1(a, al, ka) for a in grid])
+    v2 = np.array([orc.h2(a, al, ka) for a in grid])
+    assert np.all(v1 <= 1 + 1e-15) and np.all(v1 >= al - 1e-15)
+    assert np.all(v2 >= 0) and np.all(v2 <= al + 1e-15)
+    assert np.all(np.diff(v1) <= 1e-15) and np.all(np.diff(v2) >= -1e-15)   # monotone
+    assert np.max(np.abs(np.diff(v1))) < 0.02 and np.max(np.abs(np.diff(v2))) < 0.002  # continuous
+
+
+def test_weights_golden_and_constant_drift(orc, golden_dir):
+    g = read_golden(os.path.join(golden_dir, "hand_example_k2_p4.txt"))
+    for a, w1, w2 in zip(g["w_a"], g["w_h1"], g["w_h2"]):
+        assert abs(orc.h1(a, 0.1, -0.1) - w1) < 1e-12 and abs(orc.h2(a, 0.1, -0.1) - w2) < 1e-12
+    # ring example: feed u values oldest -> newest through the bookkeeping
+    st = OracleState(np.zeros(1, np.float32), 1, [(0, 1, 1)], p_hist=4, c=g["coef"], kappa=-0.1)
+    for u in g["ring"]:
+        st.norm2[:] = math.exp(2 * u)
+        h2, h1 = st.weights_next(0.1)
+    assert abs(st.last_a[0] - g["ring_a"][0]) < 1e-12
+    assert abs(h1[0] - g["ring_h1"][0]) < 1e-6 and abs(h2[0] - g["ring_h2"][0]) < 1e-7
+    # sum c_j = 1: a constant drift u_s - u_{s-1} = delta gives a = delta
+    st = OracleState(np.zeros(1, np.float32), 1, [(0, 1, 1)])
+    for s in range(8):
+        st.norm2[:] = math.exp(2 * (0.5 - 0.03 * s))
+        st.weights_next(0.1)
+    assert abs(st.last_a[0] + 0.03) < 1e-12
+
+
+def test_weights_first_sample_gives_alpha(orc):
+    # all workers start at the master (Sec. II): n2 = 0 at first, the ring is
+    # back-filled, a = 0 and both coefficients equal alpha
+    st = OracleState(np.zeros(3, np.float32), 2, [(0, 3, 1)])
+    st.norm2[:] = 0.0
+    h2, h1 = st.weights_next(0.05)
+    assert np.all(st.last_a == 0.0)
+    assert np.array_equal(h2, np.full(2, 0.05, np.float32))
+    assert np.allclose(h1, 0.05, rtol=1e-7)
+
+
+# --------------------------------------------------------------------- S5: mask
+def _mask_run(p, max_stale, T, K=8, seed=0x5EED0002):
+    st = OracleState(np.zeros(1, np.float32), K, [(0, 1, 1)])
+    return np.stack([st.mask_next(seed, t, p, max_stale) for t in range(1, T + 1)])
+
+
+def test_mask_rate_determinism_and_extremes(orc):
+    T, K = 4000, 8
+    for p in (0.1, 1 / 3, 0.25):
+        m = _mask_run(p, 1, T)
+        rate = 1.0 - m.mean()
+        assert abs(rate - p) < 5 * math.sqrt(p * (1 - p) / (T * K))
+    assert np.array_equal(_mask_run(0.2, 1, 200), _mask_run(0.2, 1, 200))
+    assert not np.array_equal(_mask_run(0.2, 1, 200), _mask_run(0.2, 1, 200, seed=7))
+    assert _mask_run(0.0, 1, 100).all()
+    assert not _mask_run(1.0, 1, 100).any()
+
+
+def test_mask_stale_durations_uniform(orc):
+    T, K = 20000, 8
+    m = _mask_run(0.05, 8, T, K)
+    runs = []
+    for i in range(K):
+        col, t = m[:, i], 0
+        while t < T:
+            if col[t] == 0:
+                s = t
+                while t < T and col[t] == 0:
+                    t += 1
+                runs.append(t - s)
+            else:
+                t += 1
+    runs = np.array(runs)
+    # outages last 1..8 rounds (longer only when two outages abut); all lengths occur
+    short = runs[runs <= 8]
+    assert len(short) > 0.7 * len(runs)
+    hist = np.bincount(short, minlength=9)[1:9]
+    assert hist.min() > 0.5 * hist.mean()
+
+
+def test_mask_threshold_by_hand(orc):
+    # worker i fails in round t iff Philox(seed; (0, i, t, 1))[0] < floor(p * 2^32)
+    seed, p = 0xABCDEF0123, 0.3
+    st = OracleState(np.zeros(1, np.float32), 5, [(0, 1, 1)])
+    for t in range(1, 30):
+        m = st.mask_next(seed, t, p, 1)
+        for i in range(5):
+            r = orc.philox([0, i, t, 1], [seed & 0xffffffff, seed >> 32])[0]
+            assert m[i] == (0 if r < math.floor(p * 2 ** 32) else 1)
+
+
+# ------------------------------------------------------------- whole rounds
+def test_hand_example_full_round(orc, golden_dir):
+    """The worked two-worker example: local step, distance, weighted exchange."""
+    g = read_golden(os.path.join(golden_dir, "hand_example_k2_p4.txt"))
+    # find a (seed, round) whose Rademacher draw equals the example's z for both workers
+    want = np.stack([g["z0"], g["z1"]]).astype(np.float32)
+    found = None
+    for seed in range(2000):
+        if np.array_equal(orc.sample_z(seed, 1, 2, 4), want):
+            found = seed
+            break
+    assert found is not None
+    st = OracleState(g["x0"].astype(np.float32), 2, [(0, 4, 2)])
+    grad = np.stack([g["g0"], g["g1"]]).astype(np.float32)
+    hvp = np.stack([g["hvp0"], g["hvp1"]]).astype(np.float32)
+    st.local_step(grad, hvp, found, 1, lr=0.1, eps=1e-4, want_dist=True)
+    tol = dict(rtol=3e-7, atol=1e-9)
+    assert np.allclose(st.m[0], g["m0"], **tol)
+    # v is quoted for beta2 = 0.999 exactly; the binary32 value of beta2 is
+    # 0.99900001287..., which scales (1 - beta2) by 0.99998713 (it cancels in v / bc2)
+    sc = (1.0 - float(np.float32(0.999))) / 0.001
+    assert np.allclose(st.v[0], g["v0"] * sc, **tol) and np.allclose(st.v[1], g["v1"] * sc, **tol)
+    assert np.allclose(st.x[0], g["x0_step"], **tol) and np.allclose(st.x[1], g["x1_step"], **tol)
+    assert np.allclose(st.norm2, g["norm2"], rtol=5e-6)
+    u = [orc.lib.orc_u_from_norm2(v) for v in st.norm2]
+    assert np.allclose(u, g["u"], atol=5e-6)
+    st.exchange(h2=g["h2"].astype(np.float32), h1=g["h1"].astype(np.float32))
+    assert np.allclose(st.center, g["center_x"], **tol)
+    assert np.allclose(st.x[0], g["x0_x"], **tol) and np.allclose(st.x[1], g["x1_x"], **tol)
+
+
+def _run_rounds(variant, K, layout_segs, P, R, tau, seed=0, p_fail=0.2, max_stale=4, frozen=True):
+    rng = np.random.default_rng(seed)
+    st = OracleState((rng.standard_normal(P) * 0.1).astype(np.float32), K, layout_segs,
+                     variant=variant)
+    pool = [(rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1),
+             rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)) for _ in range(3)]
+    alpha = min(0.05, 0.8 / K)
+    for t in range(1, R + 1):
+        mask = st.mask_next(0x5EED0002, t, p_fail, max_stale)
+        g, hv = pool[t % 3]
+        ex = t % tau == 0
+        st.local_step(g, hv, 0x5EED0001, t, lr=0.01, active=mask if frozen else None, want_dist=ex)
+        if ex:
+            h2, h1 = st.weights_next(alpha)
+            st.exchange(mask, h2, h1)
+    return st
+
+
+def test_openmp_build_is_bit_identical():
+    segs = [(0, 90, 9), (90, 30, 1), (120, 98, 49), (220, 37, 1)]
+    a = _run_rounds("fp32", 5, segs, 257, 24, 4)
+    b = _run_rounds("omp", 5, segs, 257, 24, 4)
+    for name in ("x", "m", "v", "center", "uhist", "step"):
+        assert np.array_equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_fp32_drift_against_double_arithmetic():
+    # binary32 canonical arithmetic vs the same steps in double.  The moments agree
+    # far inside the 1e-5 relative / 1e-6 absolute parity budget and so does the
+    # typical parameter; a few parameters whose sqrt(vhat) is close to eps take very
+    # large steps and amplify binary32 rounding beyond the budget.  So a second
+    # binary32 implementation can only be held to that budget if it rounds the same
+    # way, which is why the parity tests ask the device for the canonical order.
+    segs = [(0, 900, 9), (900, 124, 1), (1024, 980, 49)]
+    a = _run_rounds("fp32", 4, segs, 2004, 100, 4)
+    b = _run_rounds("fp64", 4, segs, 2004, 100, 4)
+    ratio = {}
+    for name in ("x", "m", "v", "center"):
+        va, vb = getattr(a, name).astype(np.float64), getattr(b, name).astype(np.float64)
+        ratio[name] = np.abs(va - vb) / (1e-6 + 1e-5 * np.abs(vb))
+    assert ratio["m"].max() < 0.1 and ratio["v"].max() < 0.1
+    assert np.median(ratio["x"]) < 0.1 and np.mean(ratio["x"] > 1) < 0.2
+    assert np.median(ratio["center"]) < 0.2
+
+
+def test_round_driver_brute_force_tiny():
+    """K=2, P=6, two rounds and an exchange re-derived with Python floats in the order
+    the paper's equations are applied; binary32 rounding emulated with numpy scalars."""
+    f = np.float32
+    K, P = 2, 6
+    segs = [(0, 4, 2), (4, 2, 1)]
+    o = oracle.load("fp32")
+    rng = np.random.default_rng(12)
+    c0 = rng.standard_normal(P).astype(f)
+    st = OracleState(c0, K, segs)
+    x = [[f(v) for v in c0] for _ in range(K)]
+    m = [[f(0)] * P for _ in range(K)]
+    v = [[f(0)] * P for _ in range(K)]
+    c = [f(v_) for v_ in c0]
+    b1, b2, lr, eps = f(0.9), f(0.999), f(0.05), f(1e-4)
+    for t in (1, 2):
+        g = rng.standard_normal((K, P)).astype(f)
+        hv = rng.standard_normal((K, P)).astype(f)
+        st.local_step(g, hv, 77, t, lr=float(lr), want_dist=(t == 2))
+        z = o.sample_z(77, t, K, P)
+        for i in range(K):
+            d = [f(z[i, j] * hv[i, j]) for j in range(P)]
+            dbar = list(d)
+            for q in (0, 2):
+                mean = f(f(d[q] + d[q + 1]) / f(2))
+                dbar[q] = dbar[q + 1] = mean
+            bc1 = f(1.0 - float(b1) ** t)
+            bc2 = f(1.0 - float(b2) ** t)
+            for j in range(P):
+                m[i][j] = f(f(b1 * m[i][j]) + f(f(f(1) - b1) * g[i, j]))
+                v[i][j] = f(f(b2 * v[i][j]) + f(f(f(f(1) - b2) * dbar[j]) * dbar[j]))
+                den = f(np.sqrt(f(v[i][j] / bc2)) + eps)
+                x[i][j] = f(x[i][j] - f(lr * f(f(m[i][j] / bc1) / den)))
+    assert np.array_equal(st.x, np.array(x, f)) and np.array_equal(st.v, np.array(v, f))
+    h2 = np.array([0.05, 0.02], f)
+    h1 = np.array([0.05, 0.6], f)
+    st.exchange(h2=h2, h1=h1)
+    for j in range(P):
+        acc = f(0)
+        for i in range(K):
+            d = f(x[i][j] - c[j])
+            acc = f(acc + f(h2[i] * d))
+            x[i][j] = f(x[i][j] - f(h1[i] * d))
+        c[j] = f(c[j] + acc)
+    assert np.array_equal(st.x, np.array(x, f)) and np.array_equal(st.center, np.array(c, f))
