@@ -1,0 +1,235 @@
+/*
+ * adahess.h - C ABI of the batched AdaHessian + elastic-averaging round on one GPU.
+ *
+ * The library keeps K simulated workers and one master of a data-parallel system
+ * (Xu & Carr, "A Dynamic Weighting Strategy to Mitigate Worker Node Failure in
+ * Distributed Deep Learning", Sec. II: one master, several workers, each starting
+ * as a copy of the master) as a batched [K, P] binary32 state in device memory:
+ *
+ *     x[K][P]  worker parameters      m[K][P]  first moment (EMA of the gradient)
+ *     c[P]     master parameters      v[K][P]  second moment (EMA of the squared,
+ *                                              spatially averaged Hessian diagonal)
+ *
+ * One *round* is one local AdaHessian step of every active worker
+ * (ah_local_step); every tau-th round the caller also runs the elastic exchange
+ * with the master (easgd_exchange), with per-worker coefficients from the dynamic
+ * weighting rule (dw_weights_next) and a seeded failure mask (dw_mask_next).
+ *
+ * Conventions
+ *   - Every function returns an int status: AH_OK (0) or a negative AH_ERR_* code.
+ *     Nothing throws, aborts or traps across this boundary.
+ *   - "device pointer" = memory of the handle's CUDA device; "host pointer" =
+ *     ordinary host memory.  Host arrays are copied during the call and may be
+ *     reused as soon as it returns.
+ *   - All kernels are enqueued on the handle's stream and the calls return without
+ *     waiting, except where a function is marked "synchronises".
+ *   - A handle must not be used from two threads at once.
+ *   - Arithmetic: IEEE binary32, round-to-nearest, one rounding per operation in
+ *     the order the formulas below are written (no fused multiply-add).
+ */
+#ifndef ADAHESS_H_
+#define ADAHESS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes -------------------------------------------------------- */
+#define AH_OK                 0
+#define AH_ERR_INVALID_ARG   (-1)  /* null pointer, K/P/period out of range, bad enum      */
+#define AH_ERR_ALIGN         (-2)  /* device pointer not 16-byte aligned, or ld % 4 != 0    */
+#define AH_ERR_SEGMENTS      (-3)  /* segment table unsorted, overlapping, out of range,
+                                      block > AH_MAX_BLOCK, or length % block != 0         */
+#define AH_ERR_ALLOC         (-4)  /* device or host allocation failed / workspace too small */
+#define AH_ERR_CUDA          (-5)  /* a CUDA runtime call failed; see ah_last_cuda_error    */
+#define AH_ERR_STATE         (-6)  /* call out of order (e.g. weights asked for before a
+                                      step with want_dist = 1 produced the distances)      */
+#define AH_ERR_INTERNAL      (-7)  /* the device status word was set by a kernel            */
+
+#define AH_MAX_WORKERS  256        /* K <= 256                                              */
+#define AH_MAX_BLOCK    256        /* spatial block kh*kw <= 256                            */
+#define AH_MAX_HIST     32         /* history depth p of the raw score <= 32                */
+#define AH_ROUND_AUTO   0xFFFFFFFFu
+#define AH_DEVICE_NONE  (-2)       /* ah_alloc.device: bookkeeping-only handle, no GPU      */
+
+/* ---- types ---------------------------------------------------------------- */
+typedef struct ah_ctx ah_ctx;      /* opaque; created by ah_init, freed by ah_destroy       */
+
+/* One parameter tensor inside the flat parameter row: elements
+ * [offset, offset + length).  block = kh*kw for a convolution kernel stored
+ * [c_out][c_in][kh][kw] (each filter is one run of `block` consecutive entries over
+ * which the Hessian diagonal is averaged), 1 for any other tensor.  Segments must
+ * be sorted by offset and disjoint; indices covered by no segment behave as
+ * block = 1.  length must be a multiple of block.  flags: reserved, 0. */
+typedef struct {
+    uint64_t offset;
+    uint64_t length;
+    uint32_t block;
+    uint32_t flags;
+} ah_segment;
+
+/* Hyper-parameters of one local step. */
+typedef struct {
+    float lr;             /* eta                                                            */
+    float beta1, beta2;   /* EMA rates of the first and second moment                       */
+    float eps;            /* added to the denominator                                       */
+    float hessian_power;  /* k: denominator is (sqrt(vhat))^k + eps; 1 and 0.5 are exact    */
+    float weight_decay;   /* 0 = none; else the step direction gains weight_decay * x       */
+    uint32_t round;       /* index t of the Rademacher stream; AH_ROUND_AUTO = the handle's
+                             own 1-based count of ah_local_step calls                       */
+    const uint8_t *active;/* host pointer, K bytes, or NULL (all active): 0 = worker i
+                             skips this step entirely (its x, m, v, step count stay)        */
+    int want_dist;        /* 1 = also compute n2_i = ||x_i - c||^2 after the step, for all
+                             K workers, into the handle (read by dw_weights_next)           */
+} ah_hyper;
+
+/* Optional placement: caller-owned device memory and stream.  workspace must be
+ * 256-byte aligned, at least ah_workspace_bytes() long, and outlive the handle; the
+ * library never frees it.  With opt == NULL the handle allocates its own memory
+ * with cudaMalloc on the current device and uses the default stream. */
+typedef struct {
+    void  *workspace;        /* device pointer or NULL (= allocate)                         */
+    size_t workspace_bytes;
+    void  *cuda_stream;      /* cudaStream_t, or NULL for the default stream                */
+    int    device;           /* CUDA device ordinal, -1 for the current device, or
+                                AH_DEVICE_NONE: a handle that holds no device state and
+                                makes no CUDA call.  It serves only the host-side
+                                bookkeeping (dw_config, dw_mask_next,
+                                dw_weights_from_norm2, the host selectors of
+                                ah_state_get/set), e.g. on a coordinator without a GPU;
+                                every other call returns AH_ERR_STATE.                  */
+} ah_alloc;
+
+/* Which part of the state ah_state_get / ah_state_set address. */
+enum {
+    AH_X = 0,          /* float  [K][P] (worker = -1) or [P] (worker = i)                   */
+    AH_M = 1,          /* same shape                                                        */
+    AH_V = 2,          /* same shape                                                        */
+    AH_CENTER = 3,     /* float  [P]   master parameters (worker ignored)                   */
+    AH_NORM2 = 4,      /* double [K]   last ||x_i - c||^2 (host side only)                  */
+    AH_STEP = 5,       /* uint32 [K]   steps taken by each worker (host side only)          */
+    AH_UHIST = 6,      /* double [K][p+1] ring of u_i, newest first (host side only)        */
+    AH_DOWN_UNTIL = 7, /* uint32 [K]   first round at which each worker is up again (host)  */
+    AH_ROUND = 8,      /* uint32 [2]   {calls to ah_local_step, ring filled flag} (host)    */
+    AH_INFO = 9,       /* uint32 [4]   {tiles, runs, elements per tile, row stride} (get only)  */
+    AH_RUNS = 10,      /* uint32 [runs][4]  {start, end, block, reciprocal}: the row cut into
+                          maximal runs of equal spatial block (get only, host)              */
+    AH_TILES = 11      /* uint32 [tiles][4] {first run, e0, e1, flags}: each tile's range
+                          widened to whole spatial blocks [e0, e1); flags bit 0 = the tile
+                          touches a block > 1 (get only, host)                              */
+};
+
+/* ---- life cycle ------------------------------------------------------------ */
+
+/* Bytes of device workspace a handle for (K, P) with nseg segments needs.
+ * Host-only arithmetic; touches no GPU. */
+int ah_workspace_bytes(int K, uint64_t P, int nseg, size_t *out);
+
+/* Create a handle for K workers of P parameters each (Sec. II set-up).
+ *   segs/nseg : host pointer to the tensor table (copied); nseg may be 0.
+ *   opt       : optional placement, may be NULL.
+ * On return m = v = 0, step counts = 0, x and c are zero: load the master with
+ * ah_state_set(AH_CENTER) and call ah_broadcast_center.  1 <= K <= AH_MAX_WORKERS,
+ * 1 <= P < 2^31.  Errors: INVALID_ARG, SEGMENTS, ALLOC, CUDA. */
+int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg,
+            const ah_alloc *opt);
+
+/* Free the handle and any memory it allocated itself.  Synchronises. NULL is OK. */
+int ah_destroy(ah_ctx *h);
+
+/* Copy state in / out.  `which` is one of the AH_* selectors above; `worker` picks
+ * one row of AH_X/AH_M/AH_V or is -1 for all K rows packed as [K][P].  For the
+ * float selectors the other side may be a device pointer (on_device = 1) or a
+ * host pointer (0); the host-side selectors (AH_NORM2 ... AH_ROUND) take host
+ * pointers only.  ah_state_get synchronises the handle's stream; ah_state_set is
+ * ordered after earlier work on the stream and returns when the copy is done.
+ * Together they give an exact snapshot for checkpoint and resume. */
+int ah_state_set(ah_ctx *h, int which, int worker, const void *src, int src_on_device);
+int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device);
+
+/* x_i <- c for every worker: each worker starts as a copy of the master (Sec. II). */
+int ah_broadcast_center(ah_ctx *h);
+
+/* ---- the round --------------------------------------------------------------- */
+
+/* Rademacher vectors of round `round` (Sec. IV-B, Hutchinson's method) as +-1.0f:
+ * dst[i*ld + j] = z_{round,i,j}, device pointer, ld >= P.  z is a pure function
+ * of (z_seed, round, i, j): Philox4x32-10 with key (z_seed low, z_seed high) and
+ * counter (j >> 7, i, round, 0); element j reads bit (j & 31) of output word
+ * (j >> 5) & 3; bit 0 -> +1, bit 1 -> -1.  A caller forms the Hessian-vector
+ * product Hz with this z and hands it to ah_local_step, which regenerates the same
+ * z internally (no z buffer is read there). */
+int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t ld);
+
+/* One local AdaHessian step of every active worker (Sec. IV-B; Eq. 4), fused in
+ * one pass over the state.  For worker i with t_i = its step count after this step:
+ *     D      = z (.) hvp                     Hutchinson estimate, one sample
+ *     Dbar   = block mean of D               spatial averaging inside each tensor,
+ *                                            summed in ascending index order
+ *     m      = beta1*m + (1-beta1)*grad
+ *     v      = beta2*v + ((1-beta2)*Dbar)*Dbar
+ *     mhat   = m / (1-beta1^t_i),  vhat = v / (1-beta2^t_i)
+ *     x      = x - lr * ( mhat / ((sqrt vhat)^k + eps)  [+ weight_decay * x] )
+ * grad, hvp: device pointers, [K][ld] row-major, ld >= P, ld % 4 == 0, 16-byte
+ * aligned, read only, must stay valid until the stream has run the step.
+ * With hy->want_dist the squared distances ||x_i - c||^2 (binary32 difference,
+ * squared and summed in double, pairwise order) are left in the handle.
+ * Errors: INVALID_ARG, ALIGN, CUDA. */
+int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
+                  uint64_t z_seed, const ah_hyper *hy);
+
+/* Parameters of the dynamic weighting rule (Sec. V-B): history depth p, the
+ * coefficients c_0..c_{p-1} of Eqs. 10-11 (c_0 weighs the newest difference; they
+ * should sum to 1) and the threshold kappa < 0 of h1/h2.  Defaults set by ah_init:
+ * p = 4, c = (0.4, 0.3, 0.2, 0.1), kappa = -0.1.  Clears the history. */
+int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa);
+
+/* Dynamic weights for the coming exchange (Sec. V-B).  Synchronises (waits for the
+ * distances of the last want_dist step).  For each worker: u = log||x_i - c||,
+ * pushed into its history ring (the first sample fills the ring);
+ *     a  = sum_{j<p} c_j (u_{s-j} - u_{s-j-1})                       Eqs. 10-11
+ *     h1 = 1 if a < kappa;  1 + ((1-alpha)/kappa)(a - kappa) if a <= 0;  else alpha
+ *     h2 = 0 if a < kappa;  (-alpha/kappa) a + alpha          if a <= 0;  else alpha
+ * weights: host pointer, 2K floats: h2[0..K) (master-side coefficients) followed by
+ * h1[0..K) (worker-side).  Errors: STATE when no distances are pending. */
+int dw_weights_next(ah_ctx *h, float alpha, float *weights);
+
+/* The same rule with the squared distances supplied by the caller (host pointer, K
+ * doubles) instead of taken from the last want_dist step: for callers that assemble
+ * ||x_i - c||^2 themselves, e.g. from column shards held by several GPUs.
+ * Touches no GPU. */
+int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *weights);
+
+/* Seeded failure / straggler mask for round `round` (Sec. VI: communication between
+ * a worker and the master is suppressed part of the time).  mask[i] = 1: worker i
+ * is up.  A worker that is up fails with probability p_fail (Philox draw keyed on
+ * (seed; i, round)); a failure lasts 1 round if max_stale == 1, else a uniform
+ * 1..max_stale rounds.  mask: host pointer, K bytes.  Host-only; touches no GPU. */
+int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int max_stale,
+                 uint8_t *mask);
+
+/* Weighted elastic exchange (Eqs. 12-13; with equal coefficients the EASGD pull of
+ * Eqs. 8-9), all workers seeing the same old master value.  For every column j:
+ *     c = center_j;  acc = 0
+ *     for i = 0..K-1 with worker_mask[i] != 0:
+ *         d = x_ij - c;   acc += h2_i * d;   x_ij -= h1_i * d
+ *     center_j = c + acc
+ * worker_mask: host pointer, K bytes, or NULL (all workers take part).
+ * weights: host pointer, 2K floats as written by dw_weights_next, or NULL
+ * (h1_i = h2_i = alpha for all i).  alpha is ignored when weights != NULL. */
+int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha);
+
+/* ---- diagnostics ------------------------------------------------------------- */
+const char *ah_status_string(int status);
+/* cudaError_t of the last failed runtime call on this handle (0 if none). */
+int ah_last_cuda_error(const ah_ctx *h);
+/* Number of kernel launches this handle has enqueued since ah_init. */
+uint64_t ah_launch_count(const ah_ctx *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAHESS_H_ */

@@ -1,0 +1,555 @@
+// Host side of the AdaHessian + elastic-averaging library: the handle, argument
+// checks, workspace layout, the per-tile tensor descriptors, and the O(K) weight and
+// failure bookkeeping of the dynamic weighting rule.  Kernels live in ah_kernels.cu.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "ah_internal.h"
+
+using namespace ah;
+
+struct ah_ctx {
+    int K = 0;
+    uint32_t P = 0;
+    uint64_t lds = 0;              // row stride of x, m, v, c (P rounded up to 4)
+    uint32_t ntiles = 0, ntiles_pad = 0;
+    int device = 0;
+    bool has_device = true;        // false: bookkeeping-only handle (AH_DEVICE_NONE)
+    std::vector<Run> runs_host;
+    std::vector<TileInfo> tiles_host;
+    cudaStream_t stream = nullptr;
+    bool owns_workspace = false;
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
+
+    // device views into the workspace
+    float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
+    double *partials = nullptr, *scratch = nullptr, *norm2_dev = nullptr;
+    Run *runs = nullptr;
+    TileInfo *tiles = nullptr;
+    uint32_t nruns = 0;
+
+    // host state
+    double *norm2_host = nullptr;  // pinned, K doubles
+    cudaEvent_t norm2_ready = nullptr;
+    bool norm2_pending = false;    // a want_dist step has been enqueued since the last read
+    double norm2_last[AH_MAX_WORKERS];
+    uint32_t step[AH_MAX_WORKERS];
+    uint32_t down_until[AH_MAX_WORKERS];
+    uint32_t calls = 0;            // ah_local_step calls so far
+    int p_hist = 4;
+    double coef[AH_MAX_HIST];
+    double kappa = -0.1;
+    std::vector<double> uhist;     // [K][p_hist + 1], newest first
+    int ring_filled = 0;
+
+    int last_cuda = 0;
+    uint64_t launches = 0;
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline uint32_t pow2_at_least(uint32_t n)
+{
+    uint32_t p = 1;
+    while (p < n) p <<= 1;
+    return p;
+}
+
+int cuda_fail(ah_ctx *h, cudaError_t e)
+{
+    if (h) h->last_cuda = (int)e;
+    return AH_ERR_CUDA;
+}
+
+#define AH_CUDA(h, call)                                    \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail((h), e_);   \
+    } while (0)
+
+struct Layout {
+    size_t x, m, v, c, partials, scratch, norm2, runs, tiles, total;
+};
+
+// Offsets of every array inside the workspace (each 256-byte aligned).
+Layout workspace_layout(int K, uint64_t P, int nruns_max)
+{
+    const uint64_t lds = (P + 3) / 4 * 4;
+    const uint32_t ntiles = (uint32_t)((P + kTile - 1) / kTile);
+    const uint32_t ntp = pow2_at_least(ntiles);
+    Layout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.x = take((size_t)K * lds * sizeof(float));
+    L.m = take((size_t)K * lds * sizeof(float));
+    L.v = take((size_t)K * lds * sizeof(float));
+    L.c = take((size_t)lds * sizeof(float));
+    L.partials = take((size_t)K * ntp * sizeof(double));
+    L.scratch = take((size_t)K * ntp * sizeof(double));
+    L.norm2 = take((size_t)AH_MAX_WORKERS * sizeof(double));
+    L.runs = take((size_t)nruns_max * sizeof(Run));
+    L.tiles = take((size_t)ntiles * sizeof(TileInfo));
+    L.total = off;
+    return L;
+}
+
+// Cut [0, P) into maximal runs of equal spatial block; gaps behave as block 1.
+int build_runs(uint64_t P, const ah_segment *segs, int nseg, std::vector<Run> &runs)
+{
+    runs.clear();
+    auto push = [&](uint64_t a, uint64_t b, uint32_t block) {
+        if (a >= b) return;
+        if (!runs.empty() && runs.back().block == 1 && block == 1 && runs.back().end == a) {
+            runs.back().end = (uint32_t)b;
+            return;
+        }
+        Run r;
+        r.start = (uint32_t)a;
+        r.end = (uint32_t)b;
+        r.block = block;
+        r.magic = block > 1 ? (uint32_t)(((1ull << 32) + block - 1) / block) : 0u;
+        runs.push_back(r);
+    };
+    uint64_t pos = 0;
+    for (int s = 0; s < nseg; ++s) {
+        const ah_segment &g = segs[s];
+        if (g.block < 1 || g.block > AH_MAX_BLOCK) return AH_ERR_SEGMENTS;
+        if (g.offset < pos || g.offset > P || g.length > P - g.offset) return AH_ERR_SEGMENTS;
+        if (g.length % g.block != 0) return AH_ERR_SEGMENTS;
+        push(pos, g.offset, 1);
+        push(g.offset, g.offset + g.length, g.block);
+        pos = g.offset + g.length;
+    }
+    push(pos, P, 1);
+    return AH_OK;
+}
+
+void build_tiles(uint32_t P, const std::vector<Run> &runs, std::vector<TileInfo> &tiles)
+{
+    const uint32_t ntiles = (P + kTile - 1) / kTile;
+    tiles.resize(ntiles);
+    size_t ri = 0;
+    for (uint32_t t = 0; t < ntiles; ++t) {
+        const uint32_t t0 = t * (uint32_t)kTile;
+        const uint32_t t1 = (uint64_t)t0 + kTile < P ? t0 + kTile : P;
+        while (runs[ri].end <= t0) ++ri;
+        TileInfo ti;
+        ti.run0 = (uint32_t)ri;
+        const Run &first = runs[ri];
+        ti.e0 = first.block > 1 ? first.start + (t0 - first.start) / first.block * first.block : t0;
+        size_t rj = ri;
+        uint32_t flags = 0;
+        for (;;) {
+            if (runs[rj].block > 1) flags |= 1u;
+            if (runs[rj].end >= t1) break;
+            ++rj;
+        }
+        const Run &last = runs[rj];
+        ti.e1 = last.block > 1
+                    ? last.start + ((t1 - 1 - last.start) / last.block + 1) * last.block
+                    : t1;
+        ti.flags = flags;
+        tiles[t] = ti;
+    }
+}
+
+void reset_history(ah_ctx *h)
+{
+    h->uhist.assign((size_t)h->K * (size_t)(h->p_hist + 1), 0.0);
+    h->ring_filled = 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ah_workspace_bytes(int K, uint64_t P, int nseg, size_t *out)
+{
+    if (!out || K < 1 || K > AH_MAX_WORKERS || P < 1 || P >= (1ull << 31) || nseg < 0)
+        return AH_ERR_INVALID_ARG;
+    *out = workspace_layout(K, P, 2 * nseg + 1).total;
+    return AH_OK;
+}
+
+int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, const ah_alloc *opt)
+{
+    if (!out) return AH_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (K < 1 || K > AH_MAX_WORKERS || P < 1 || P >= (1ull << 31) || nseg < 0 || (nseg > 0 && !segs))
+        return AH_ERR_INVALID_ARG;
+
+    std::vector<Run> runs;
+    int rc = build_runs(P, segs, nseg, runs);
+    if (rc != AH_OK) return rc;
+    std::vector<TileInfo> tiles;
+    build_tiles((uint32_t)P, runs, tiles);
+
+    ah_ctx *h = new (std::nothrow) ah_ctx();
+    if (!h) return AH_ERR_ALLOC;
+    h->K = K;
+    h->P = (uint32_t)P;
+    h->lds = (P + 3) / 4 * 4;
+    h->ntiles = (uint32_t)tiles.size();
+    h->ntiles_pad = pow2_at_least(h->ntiles);
+    h->nruns = (uint32_t)runs.size();
+    memset(h->step, 0, sizeof(h->step));
+    memset(h->down_until, 0, sizeof(h->down_until));
+    memset(h->norm2_last, 0, sizeof(h->norm2_last));
+    const double c_default[4] = {0.4, 0.3, 0.2, 0.1};
+    memcpy(h->coef, c_default, sizeof(c_default));
+    reset_history(h);
+
+    h->runs_host = runs;
+    h->tiles_host = tiles;
+    if (opt && opt->device == AH_DEVICE_NONE) {
+        h->has_device = false;
+        *out = h;
+        return AH_OK;
+    }
+
+    auto fail = [&](int code) { ah_destroy(h); return code; };
+
+    cudaError_t e;
+    if (opt && opt->device >= 0) {
+        h->device = opt->device;
+        if ((e = cudaSetDevice(h->device)) != cudaSuccess) { h->last_cuda = (int)e; return fail(AH_ERR_CUDA); }
+    } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
+        h->last_cuda = (int)e;
+        return fail(AH_ERR_CUDA);
+    }
+    h->stream = opt ? (cudaStream_t)opt->cuda_stream : nullptr;
+
+    const Layout L = workspace_layout(K, P, 2 * nseg + 1);
+    h->workspace_bytes = L.total;
+    if (opt && opt->workspace) {
+        if (((uintptr_t)opt->workspace & 255u) != 0) return fail(AH_ERR_ALIGN);
+        if (opt->workspace_bytes < L.total) return fail(AH_ERR_ALLOC);
+        h->workspace = opt->workspace;
+    } else {
+        if ((e = cudaMalloc(&h->workspace, L.total)) != cudaSuccess) {
+            h->last_cuda = (int)e;
+            h->workspace = nullptr;
+            return fail(AH_ERR_ALLOC);
+        }
+        h->owns_workspace = true;
+    }
+    char *base = (char *)h->workspace;
+    h->x = (float *)(base + L.x);
+    h->m = (float *)(base + L.m);
+    h->v = (float *)(base + L.v);
+    h->c = (float *)(base + L.c);
+    h->partials = (double *)(base + L.partials);
+    h->scratch = (double *)(base + L.scratch);
+    h->norm2_dev = (double *)(base + L.norm2);
+    h->runs = (Run *)(base + L.runs);
+    h->tiles = (TileInfo *)(base + L.tiles);
+
+    if ((e = cudaMallocHost((void **)&h->norm2_host, AH_MAX_WORKERS * sizeof(double))) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->norm2_ready, cudaEventDisableTiming)) != cudaSuccess) {
+        h->last_cuda = (int)e;
+        return fail(AH_ERR_ALLOC);
+    }
+    // state (and its row padding) starts at zero; descriptors go up once
+    if ((e = cudaMemsetAsync(h->workspace, 0, L.runs, h->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(h->runs, runs.data(), runs.size() * sizeof(Run), cudaMemcpyHostToDevice,
+                             h->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(h->tiles, tiles.data(), tiles.size() * sizeof(TileInfo),
+                             cudaMemcpyHostToDevice, h->stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(h->stream)) != cudaSuccess) {
+        h->last_cuda = (int)e;
+        return fail(AH_ERR_CUDA);
+    }
+    *out = h;
+    return AH_OK;
+}
+
+int ah_destroy(ah_ctx *h)
+{
+    if (!h) return AH_OK;
+    int rc = AH_OK;
+    if (h->has_device && (h->workspace || h->norm2_host)) {
+        cudaError_t e = cudaStreamSynchronize(h->stream);
+        if (e != cudaSuccess) rc = AH_ERR_CUDA;
+    }
+    if (h->norm2_ready) cudaEventDestroy(h->norm2_ready);
+    if (h->norm2_host) cudaFreeHost(h->norm2_host);
+    if (h->owns_workspace && h->workspace) cudaFree(h->workspace);
+    delete h;
+    return rc;
+}
+
+int ah_broadcast_center(ah_ctx *h)
+{
+    if (!h) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    AH_CUDA(h, launch_broadcast(h->x, h->c, h->lds, h->K, h->stream));
+    h->launches += 1;
+    return AH_OK;
+}
+
+int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t ld)
+{
+    if (!h || !dst || ld < h->P) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    AH_CUDA(h, launch_sample_z(dst, ld, h->P, h->K, (uint32_t)(z_seed & 0xffffffffu),
+                               (uint32_t)(z_seed >> 32), round, h->stream));
+    h->launches += 1;
+    return AH_OK;
+}
+
+int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
+                  const ah_hyper *hy)
+{
+    if (!h || !grad || !hvp || !hy || ld < h->P) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    if (!(hy->beta1 >= 0.f && hy->beta1 < 1.f && hy->beta2 >= 0.f && hy->beta2 < 1.f))
+        return AH_ERR_INVALID_ARG;
+    if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0 || ((uintptr_t)hvp & 15u) != 0)
+        return AH_ERR_ALIGN;
+
+    StepParams p;
+    p.x = h->x; p.m = h->m; p.v = h->v; p.c = h->c;
+    p.grad = grad; p.hvp = hvp;
+    p.partials = h->partials;
+    p.runs = h->runs; p.tiles = h->tiles;
+    p.lds = h->lds; p.ld = ld;
+    p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
+    p.key0 = (uint32_t)(z_seed & 0xffffffffu);
+    p.key1 = (uint32_t)(z_seed >> 32);
+    h->calls += 1;
+    p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
+    p.lr = hy->lr; p.beta1 = hy->beta1; p.beta2 = hy->beta2;
+    p.omb1 = 1.0f - hy->beta1;
+    p.omb2 = 1.0f - hy->beta2;
+    p.eps = hy->eps; p.hpow = hy->hessian_power; p.wd = hy->weight_decay;
+    for (int i = 0; i < h->K; ++i) {
+        const bool on = !hy->active || hy->active[i] != 0;
+        p.active[i] = on ? 1 : 0;
+        if (on) h->step[i] += 1;
+        // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
+        // (a worker that sat out steps has taken fewer); double, then one rounding
+        const double t = (double)(h->step[i] ? h->step[i] : 1u);
+        p.bc1[i] = (float)(1.0 - pow((double)hy->beta1, t));
+        p.bc2[i] = (float)(1.0 - pow((double)hy->beta2, t));
+    }
+    const bool dist = hy->want_dist != 0;
+    AH_CUDA(h, launch_local_step(p, h->K, dist, h->stream));
+    h->launches += 1;
+    if (dist) {
+        AH_CUDA(h, launch_norm2_finalize(h->partials, h->scratch, h->ntiles, h->ntiles_pad, h->K,
+                                         h->norm2_dev, h->stream));
+        h->launches += 1;
+        AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, h->K * sizeof(double),
+                                   cudaMemcpyDeviceToHost, h->stream));
+        AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
+        h->norm2_pending = true;
+    }
+    return AH_OK;
+}
+
+// ---- state in / out -----------------------------------------------------------
+static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_device, bool to_user)
+{
+    if (!h || !user) return AH_ERR_INVALID_ARG;
+    const size_t row = (size_t)h->P * sizeof(float);
+    if (which == AH_X || which == AH_M || which == AH_V || which == AH_CENTER) {
+        if (!h->has_device) return AH_ERR_STATE;
+        float *base = which == AH_X ? h->x : which == AH_M ? h->m : which == AH_V ? h->v : h->c;
+        size_t rows = 1;
+        if (which != AH_CENTER) {
+            if (worker < -1 || worker >= h->K) return AH_ERR_INVALID_ARG;
+            if (worker >= 0) base += (size_t)worker * h->lds;
+            else rows = (size_t)h->K;
+        }
+        const size_t pitch = (size_t)h->lds * sizeof(float);
+        cudaMemcpyKind kind;
+        if (to_user) kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost;
+        else         kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+        if (to_user) AH_CUDA(h, cudaMemcpy2DAsync(user, row, base, pitch, row, rows, kind, h->stream));
+        else         AH_CUDA(h, cudaMemcpy2DAsync(base, pitch, user, row, row, rows, kind, h->stream));
+        AH_CUDA(h, cudaStreamSynchronize(h->stream));
+        return AH_OK;
+    }
+    if (on_device) return AH_ERR_INVALID_ARG;
+    void *ptr;
+    size_t bytes;
+    uint32_t round_info[2];
+    uint32_t info[4];
+    if ((which == AH_INFO || which == AH_RUNS || which == AH_TILES) && !to_user)
+        return AH_ERR_INVALID_ARG;
+    switch (which) {
+    case AH_INFO:
+        info[0] = h->ntiles; info[1] = h->nruns; info[2] = (uint32_t)kTile; info[3] = (uint32_t)h->lds;
+        ptr = info; bytes = sizeof(info);
+        break;
+    case AH_RUNS:  ptr = h->runs_host.data(); bytes = h->runs_host.size() * sizeof(Run); break;
+    case AH_TILES: ptr = h->tiles_host.data(); bytes = h->tiles_host.size() * sizeof(TileInfo); break;
+    case AH_NORM2:      ptr = h->norm2_last; bytes = h->K * sizeof(double); break;
+    case AH_STEP:       ptr = h->step; bytes = h->K * sizeof(uint32_t); break;
+    case AH_UHIST:      ptr = h->uhist.data(); bytes = h->uhist.size() * sizeof(double); break;
+    case AH_DOWN_UNTIL: ptr = h->down_until; bytes = h->K * sizeof(uint32_t); break;
+    case AH_ROUND:
+        round_info[0] = h->calls;
+        round_info[1] = (uint32_t)h->ring_filled;
+        ptr = round_info; bytes = sizeof(round_info);
+        break;
+    default: return AH_ERR_INVALID_ARG;
+    }
+    if (to_user) {
+        if (which == AH_NORM2 && h->norm2_pending) {
+            AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
+            memcpy(h->norm2_last, h->norm2_host, h->K * sizeof(double));
+        }
+        memcpy(user, ptr, bytes);
+    } else {
+        memcpy(ptr, user, bytes);
+        if (which == AH_ROUND) {
+            h->calls = round_info[0];
+            h->ring_filled = (int)round_info[1];
+        }
+        if (which == AH_NORM2) h->norm2_pending = false;
+    }
+    return AH_OK;
+}
+
+int ah_state_set(ah_ctx *h, int which, int worker, const void *src, int src_on_device)
+{
+    return state_copy(h, which, worker, const_cast<void *>(src), src_on_device, false);
+}
+
+int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device)
+{
+    if (h && h->has_device) AH_CUDA(h, cudaStreamSynchronize(h->stream));
+    return state_copy(h, which, worker, dst, dst_on_device, true);
+}
+
+// ---- dynamic weights (Sec. V-B) ------------------------------------------------
+int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
+{
+    if (!h || !c || p_hist < 1 || p_hist > AH_MAX_HIST || !(kappa < 0.0)) return AH_ERR_INVALID_ARG;
+    h->p_hist = p_hist;
+    for (int j = 0; j < p_hist; ++j) h->coef[j] = c[j];
+    h->kappa = kappa;
+    reset_history(h);
+    return AH_OK;
+}
+
+int dw_weights_next(ah_ctx *h, float alpha, float *weights)
+{
+    if (!h || !weights) return AH_ERR_INVALID_ARG;
+    if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
+    AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
+    h->norm2_pending = false;
+    return dw_weights_from_norm2(h, h->norm2_host, alpha, weights);
+}
+
+int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *weights)
+{
+    if (!h || !norm2 || !weights) return AH_ERR_INVALID_ARG;
+    memcpy(h->norm2_last, norm2, h->K * sizeof(double));
+
+    const int depth = h->p_hist + 1;
+    const double a_rate = (double)alpha, kap = h->kappa;
+    const double slope_worker = (1.0 - a_rate) / kap;    // h1 falls from 1 to alpha on [kappa, 0]
+    const double slope_master = -a_rate / kap;           // h2 rises from 0 to alpha on [kappa, 0]
+    float *to_master = weights, *to_worker = weights + h->K;
+    for (int i = 0; i < h->K; ++i) {
+        double *ring = &h->uhist[(size_t)i * depth];
+        const double n2 = h->norm2_last[i];
+        const double u = 0.5 * log(n2 > 1e-300 ? n2 : 1e-300);   // log of the 2-norm
+        if (h->ring_filled) memmove(ring + 1, ring, (size_t)h->p_hist * sizeof(double));
+        else for (int j = 1; j < depth; ++j) ring[j] = u;
+        ring[0] = u;
+        double score = 0.0;                               // Eqs. 10-11
+        for (int j = 0; j < h->p_hist; ++j) score = score + h->coef[j] * (ring[j] - ring[j + 1]);
+        double w_worker, w_master;
+        if (score < kap)        { w_worker = 1.0; w_master = 0.0; }
+        else if (score <= 0.0)  { w_worker = 1.0 + slope_worker * (score - kap);
+                                  w_master = slope_master * score + a_rate; }
+        else                    { w_worker = a_rate; w_master = a_rate; }
+        to_worker[i] = (float)w_worker;
+        to_master[i] = (float)w_master;
+    }
+    h->ring_filled = 1;
+    return AH_OK;
+}
+
+// ---- failure / straggler mask (Sec. VI) -----------------------------------------
+int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int max_stale,
+                 uint8_t *mask)
+{
+    if (!h || !mask || max_stale < 1 || !(p_fail >= 0.0)) return AH_ERR_INVALID_ARG;
+    const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
+    const bool always = p_fail >= 1.0;
+    const uint32_t threshold = always ? 0u : (uint32_t)floor(p_fail * 4294967296.0);
+    for (int i = 0; i < h->K; ++i) {
+        bool up = round >= h->down_until[i];
+        if (up) {
+            uint32_t draw[4];
+            philox4x32_10(0u, (uint32_t)i, round, kDomainFail, k0, k1, draw);
+            if (always || draw[0] < threshold) {
+                uint32_t length = 1;
+                if (max_stale > 1) {
+                    uint32_t d2[4];
+                    philox4x32_10(0u, (uint32_t)i, round, kDomainStale, k0, k1, d2);
+                    length += d2[0] % (uint32_t)max_stale;
+                }
+                h->down_until[i] = round + length;
+                up = false;
+            }
+        }
+        mask[i] = up ? 1 : 0;
+    }
+    return AH_OK;
+}
+
+// ---- elastic exchange (Eqs. 12-13) -----------------------------------------------
+int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha)
+{
+    if (!h) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    ExchangeParams p;
+    p.x = h->x; p.c = h->c; p.lds = h->lds;
+    p.nvec = (uint32_t)(h->lds / 4);
+    p.nact = 0;
+    for (int i = 0; i < h->K; ++i) {
+        if (worker_mask && !worker_mask[i]) continue;
+        p.idx[p.nact] = (uint16_t)i;
+        p.h2[p.nact] = weights ? weights[i] : alpha;
+        p.h1[p.nact] = weights ? weights[h->K + i] : alpha;
+        p.nact += 1;
+    }
+    if (p.nact == 0) return AH_OK;     // nobody reaches the master: nothing moves
+    AH_CUDA(h, launch_exchange(p, h->stream));
+    h->launches += 1;
+    return AH_OK;
+}
+
+// ---- diagnostics ------------------------------------------------------------------
+const char *ah_status_string(int status)
+{
+    switch (status) {
+    case AH_OK: return "ok";
+    case AH_ERR_INVALID_ARG: return "invalid argument";
+    case AH_ERR_ALIGN: return "pointer or stride not aligned";
+    case AH_ERR_SEGMENTS: return "bad segment table";
+    case AH_ERR_ALLOC: return "allocation failed or workspace too small";
+    case AH_ERR_CUDA: return "CUDA runtime error";
+    case AH_ERR_STATE: return "call out of order";
+    case AH_ERR_INTERNAL: return "internal device error";
+    default: return "unknown status";
+    }
+}
+
+int ah_last_cuda_error(const ah_ctx *h) { return h ? h->last_cuda : 0; }
+
+uint64_t ah_launch_count(const ah_ctx *h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,111 @@
+// Internal declarations shared by the host side (ah_host.cu) and the kernels
+// (ah_kernels.cu) of the AdaHessian + elastic-averaging library.  Not installed.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "adahess.h"
+
+namespace ah {
+
+// Tile of the flat parameter row handled by one CTA: TILE consecutive elements of
+// one worker.  A power of two, so that a tile is a subtree of the pairwise
+// summation tree used for ||x_i - c||^2.
+constexpr int kTile = 2048;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kGroupsPerWarp = kTile / 128 / kWarps;   // 128 = elements per Philox block
+static_assert(kGroupsPerWarp >= 1 && kGroupsPerWarp <= 8, "warp owns 1..8 Philox groups");
+static_assert((kGroupsPerWarp & (kGroupsPerWarp - 1)) == 0, "power of two");
+
+// Shared staging of the signed Hessian-vector tile: the tile, a halo of up to
+// AH_MAX_BLOCK - 1 elements on each side (a spatial block may straddle the tile
+// edge) and slack for rounding both ends to 16 bytes.
+constexpr int kStageFloats = kTile + 2 * AH_MAX_BLOCK + 8;
+constexpr int kStageGroups = kStageFloats / 128 + 2;
+
+// The row [0, P) cut into maximal runs of equal spatial block (gaps and block-1
+// tensors merged).  magic = ceil(2^32 / block) turns r / block into one mul-hi for
+// r * block < 2^32; unused when block == 1.
+struct Run {
+    uint32_t start;
+    uint32_t end;
+    uint32_t block;
+    uint32_t magic;
+};
+
+// Per tile: first run that intersects it, and the tile's range widened to whole
+// spatial blocks [e0, e1).  flags bit 0: some run with block > 1 intersects the tile.
+struct TileInfo {
+    uint32_t run0;
+    uint32_t e0;
+    uint32_t e1;
+    uint32_t flags;
+};
+
+struct StepParams {
+    float *x, *m, *v;
+    const float *c;
+    const float *grad, *hvp;
+    double *partials;          // [K][ntiles_pad] tile sums of (x - c)^2
+    const Run *runs;
+    const TileInfo *tiles;
+    uint64_t lds;              // row stride of x, m, v (elements, multiple of 4)
+    uint64_t ld;               // row stride of grad, hvp
+    uint32_t P;
+    uint32_t ntiles;
+    uint32_t ntiles_pad;       // power of two >= ntiles
+    uint32_t key0, key1, round;
+    float lr, beta1, beta2, omb1, omb2, eps, hpow, wd;
+    float bc1[AH_MAX_WORKERS];
+    float bc2[AH_MAX_WORKERS];
+    uint8_t active[AH_MAX_WORKERS];
+};
+
+struct ExchangeParams {
+    float *x;
+    float *c;
+    uint64_t lds;
+    uint32_t nvec;             // float4 columns (= lds / 4)
+    int nact;                  // workers taking part
+    uint16_t idx[AH_MAX_WORKERS];   // their indices, ascending
+    float h1[AH_MAX_WORKERS];       // compacted to the same order
+    float h2[AH_MAX_WORKERS];
+};
+
+// Kernel launchers (ah_kernels.cu).  Each returns the cudaError_t of the launch.
+cudaError_t launch_local_step(const StepParams &p, int K, bool want_dist, cudaStream_t s);
+cudaError_t launch_norm2_finalize(double *partials, double *scratch, uint32_t ntiles,
+                                  uint32_t ntiles_pad, int K, double *norm2, cudaStream_t s);
+cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s);
+cudaError_t launch_sample_z(float *dst, uint64_t ld, uint32_t P, int K, uint32_t key0,
+                            uint32_t key1, uint32_t round, cudaStream_t s);
+cudaError_t launch_broadcast(float *x, const float *c, uint64_t lds, int K, cudaStream_t s);
+
+// Philox4x32-10 (Salmon et al., SC'11), usable on both sides.
+__host__ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t out[4])
+{
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+#ifdef __CUDA_ARCH__
+        const uint32_t hiA = __umulhi(0xD2511F53u, c0), loA = 0xD2511F53u * c0;
+        const uint32_t hiB = __umulhi(0xCD9E8D57u, c2), loB = 0xCD9E8D57u * c2;
+#else
+        const uint64_t pa = 0xD2511F53ull * c0, pb = 0xCD9E8D57ull * c2;
+        const uint32_t hiA = (uint32_t)(pa >> 32), loA = (uint32_t)pa;
+        const uint32_t hiB = (uint32_t)(pb >> 32), loB = (uint32_t)pb;
+#endif
+        const uint32_t y0 = hiB ^ c1 ^ k0;
+        const uint32_t y2 = hiA ^ c3 ^ k1;
+        c0 = y0; c1 = loB; c2 = y2; c3 = loA;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+enum : uint32_t { kDomainZ = 0, kDomainFail = 1, kDomainStale = 2 };
+
+}  // namespace ah

@@ -1,0 +1,139 @@
+"""CPU-only tests: the C-ABI library loads and exports what include/adahess.h declares,
+argument checks, and the host-side bookkeeping (failure mask, dynamic weights, tile
+descriptors) against the oracle.  No compute call touches a GPU here."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import OracleState
+from paper_2409_09242_b200 import workloads as W
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2409_09242_b200 import build
+    build.build()
+    from paper_2409_09242_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(B):
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    declared = set()
+    for fn in os.listdir(os.path.join(root, "include")):
+        text = open(os.path.join(root, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        declared |= set(re.findall(r"\b((?:ah|dw|easgd)_[a-z0-9_]+)\s*\(", text))
+    assert {"ah_init", "ah_local_step", "easgd_exchange", "ah_state_get"} <= declared
+    lib = C.CDLL(B._build.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTS)
+
+
+def test_status_strings_and_argument_checks(B):
+    assert B.ah_status_string(0) == "ok"
+    assert "segment" in B.ah_status_string(B.AH_ERR_SEGMENTS)
+    with pytest.raises(B.AdaHessError):
+        B.ah_workspace_bytes(0, 10, 0)                     # K < 1
+    with pytest.raises(B.AdaHessError):
+        B.ah_workspace_bytes(B.AH_MAX_WORKERS + 1, 10, 0)  # K too large
+    with pytest.raises(B.AdaHessError):
+        B.ah_workspace_bytes(1, 1 << 31, 0)                # P too large
+    assert B.ah_workspace_bytes(1, (1 << 31) - 1, 0) > 3 * 4 * ((1 << 31) - 1)
+    # workspace covers x, m, v [K][P] plus the master row
+    K, P = 16, 25_557_032
+    assert B.ah_workspace_bytes(K, P, 161) >= (3 * K + 1) * P * 4
+
+
+@pytest.mark.parametrize("segs,code", [
+    ([(0, 10, 3)], "SEGMENTS"),            # length not a multiple of block
+    ([(0, 9, 9), (5, 9, 9)], "SEGMENTS"),  # overlap
+    ([(9, 9, 9), (0, 9, 9)], "SEGMENTS"),  # unsorted
+    ([(0, 200, 1)], "SEGMENTS"),           # beyond P
+    ([(0, 0, 0)], "SEGMENTS"),             # block 0
+    ([(0, 514, 257)], "SEGMENTS"),         # block above the maximum
+])
+def test_bad_segment_tables_are_rejected(B, segs, code):
+    with pytest.raises(B.AdaHessError) as e:
+        B.Handle(2, 100 if segs[0][1] != 514 else 1000, segs, host_only=True)
+    assert e.value.status == getattr(B, "AH_ERR_" + code)
+
+
+def test_bookkeeping_handle_refuses_device_calls(B):
+    h = B.Handle(2, 64, [(0, 64, 1)], host_only=True)
+    assert B.raw().ah_broadcast_center(h._h) == B.AH_ERR_STATE
+    assert B.raw().easgd_exchange(h._h, None, None, 0.1) == B.AH_ERR_STATE
+    w = (C.c_float * 4)()
+    assert B.raw().dw_weights_next(h._h, 0.1, w) == B.AH_ERR_STATE
+    h.close()
+
+
+def test_mask_matches_oracle_bit_for_bit(B):
+    for K, p, stale in ((4, 0.1, 1), (16, 0.2, 8), (64, 0.3, 1), (8, 1 / 3, 4), (3, 0.0, 1), (3, 1.0, 2)):
+        h = B.Handle(K, 8, [], host_only=True)
+        ref = OracleState(np.zeros(8, np.float32), K, [])
+        for t in range(1, 400):
+            assert np.array_equal(h.dw_mask_next(0x5EED0002, t, p, stale),
+                                  ref.mask_next(0x5EED0002, t, p, stale)), (K, p, stale, t)
+        assert np.array_equal(h.ah_state_get(B.AH_DOWN_UNTIL), ref.down_until)
+        h.close()
+
+
+def test_weights_match_oracle_bit_for_bit_given_same_distances(B):
+    rng = np.random.default_rng(0)
+    for K, alpha, p_hist, kappa in ((4, 0.05, 4, -0.1), (16, 0.1, 2, -0.05), (64, 0.0125, 6, -0.3)):
+        c = rng.dirichlet(np.ones(p_hist))
+        h = B.Handle(K, 8, [], host_only=True)
+        h.dw_config(p_hist, c, kappa)
+        ref = OracleState(np.zeros(8, np.float32), K, [], p_hist=p_hist, c=c, kappa=kappa)
+        u = rng.normal(0, 1, K)
+        for s in range(60):
+            u = u + rng.normal(0, 0.08, K) - (rng.random(K) < 0.1) * 0.3
+            n2 = np.exp(2 * u)
+            if s == 0:
+                n2[:] = 0.0                      # workers start on top of the master
+            w = h.dw_weights_from_norm2(n2, alpha)
+            ref.norm2[:] = n2
+            h2, h1 = ref.weights_next(alpha)
+            assert np.array_equal(w[:K], h2) and np.array_equal(w[K:], h1), (K, s)
+        assert np.array_equal(h.ah_state_get(B.AH_UHIST, p_hist=p_hist), ref.uhist)
+        h.close()
+
+
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "vgg16", "odd"])
+def test_tile_descriptors_cover_whole_blocks(B, name):
+    if name == "odd":
+        segs = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 256)]
+        P = 13_111
+    else:
+        layout = W.LAYOUTS[name](8)
+        segs, P = W.segments(layout), W.total_params(layout)
+    h = B.Handle(2, P, segs, host_only=True)
+    ntiles, nruns, T, lds = (int(v) for v in h.ah_state_get(B.AH_INFO))
+    runs, tiles = h.ah_state_get(B.AH_RUNS), h.ah_state_get(B.AH_TILES)
+    assert ntiles == (P + T - 1) // T and lds == (P + 3) // 4 * 4 and len(runs) == nruns
+    # runs tile [0, P) exactly, and agree with the segment table element by element
+    assert runs[0, 0] == 0 and runs[-1, 1] == P and np.array_equal(runs[1:, 0], runs[:-1, 1])
+    block_of = np.ones(P, np.int64)
+    for off, n, b in segs:
+        block_of[off:off + n] = b
+    for s, e, b, _ in runs:
+        assert np.all(block_of[s:e] == b)
+    for t in range(ntiles):
+        run0, e0, e1, flags = (int(v) for v in tiles[t])
+        t0, t1 = t * T, min(P, (t + 1) * T)
+        assert runs[run0, 0] <= t0 < runs[run0, 1]
+        assert e0 <= t0 and e1 >= t1 and e1 <= P
+        assert t0 - e0 < B.AH_MAX_BLOCK and e1 - t1 < B.AH_MAX_BLOCK
+        assert flags == int(np.any(block_of[t0:t1] > 1))
+        # [e0, e1) ends on block boundaries of the runs they fall in
+        for edge in (e0, e1):
+            r = np.searchsorted(runs[:, 1], edge, side="right" if edge == e0 else "left")
+            r = min(r, nruns - 1)
+            s, e, b, _ = (int(v) for v in runs[r])
+            assert (edge - s) % b == 0 or edge == e
+    h.close()
