@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Throughput of the AdaHessian + elastic-averaging round on B200.
+
+One *step* is one communication period of the whole hot path: tau local steps of all K
+workers (Rademacher signs, Hutchinson diagonal, spatial average, moments, update), and
+on the last of them the distances to the master, the dynamic weights, the failure mask
+and the weighted elastic exchange.  The metric is parameter updates per second,
+K * P * tau * steps / time, with the time taken on the device (CUDA events on the
+library's stream, maximum over ranks).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c1|c3|c4|c5k64|...]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+With N > 1 (launched by torchrun) every rank runs an independent replica on its own
+GPU: the path has no inter-GPU exchange step, so scaling is weak by construction.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+Z_SEED, MASK_SEED, DATA_SEED = 0x5EED0001, 0x5EED0002, 0
+
+# name -> (layout, K, tau, p_fail, max_stale, frozen stragglers)
+WORKLOADS = {
+    "c1": ("quadratic", 4, 4, 0.0, 1, False),
+    "c2": ("resnet18", 8, 4, 0.1, 1, False),
+    "c3": ("resnet50", 16, 4, 0.2, 8, True),
+    "c3tau1": ("resnet50", 16, 1, 0.2, 8, True),
+    "c3tau16": ("resnet50", 16, 16, 0.2, 8, True),
+    "c4": ("vgg16", 4, 8, 0.25, 1, False),
+    "c5k4": ("resnet50", 4, 4, 0.1, 1, False),
+    "c5k16": ("resnet50", 16, 4, 0.1, 1, False),
+    "c5k32": ("resnet50", 32, 4, 0.1, 1, False),
+    "c5k64": ("resnet50", 64, 4, 0.1, 1, False),
+}
+HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weight_decay=0.0)
+
+# DRAM bytes per parameter update of the fused local-step kernel, from one ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum over the launch / (K * P)), and the hash
+# of the kernel sources it was taken on.  Reported only while the sources are unchanged.
+NCU_TRAFFIC = {"sources_sha256": None, "dram_bytes_per_update": None}
+
+
+def kernel_sources_hash() -> str:
+    h = hashlib.sha256()
+    for fn in ("ah_kernels.cu", "ah_internal.h"):
+        with open(os.path.join(ROOT, "paper_2409_09242_b200", "csrc", fn), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def make_layout(kind):
+    from paper_2409_09242_b200 import workloads as W
+    if kind == "quadratic":
+        return W.single_segment_layout(1 << 20)
+    return W.LAYOUTS[kind]()
+
+
+def alpha_for(K):
+    return min(0.05, 0.8 / K)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        clocks, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(clocks) if clocks else None, "sm_max_mhz": mx,
+                "samples": len(clocks), "reasons": sorted(reasons)}
+
+
+def run_period(h, pool, t0, wl, events=None, stage=None):
+    """One communication period starting after round t0.  With `stage` = (host_pool,
+    dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
+    memory (the end-to-end leg).  Returns bytes moved by the local-step launches."""
+    import torch
+    _, K, tau, p_fail, max_stale, frozen = wl
+    alpha = alpha_for(K)
+    for r in range(tau):
+        t = t0 + r + 1
+        mask = h.dw_mask_next(MASK_SEED, t, p_fail, max_stale)
+        ex = r == tau - 1
+        if stage is not None:
+            host_pool, g, hv = stage
+            hg, hh = host_pool[t % len(host_pool)]
+            g.copy_(hg, non_blocking=True)
+            hv.copy_(hh, non_blocking=True)
+        else:
+            g, hv = pool[t % len(pool)]
+        if events is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
+                        **HYPER)
+        if events is not None:
+            e1.record()
+            n_act = int(mask.sum()) if frozen else K
+            events.append((e0, e1, ex, n_act))
+        if ex:
+            w = h.dw_weights_next(alpha)
+            h.easgd_exchange(mask, w, alpha)
+    return t0 + tau
+
+
+def gpu_arm(args):
+    import torch
+    from paper_2409_09242_b200 import binding, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = WORKLOADS[args.workload]
+    kind, K, tau, p_fail, max_stale, frozen = wl
+    layout = make_layout(kind)
+    segs, P = W.segments(layout), W.total_params(layout)
+    ld = W.padded_ld(P)
+    dev = torch.device("cuda", local_rank)
+
+    # synthetic inputs, resident in HBM before the timed region
+    pair_bytes = 2 * K * ld * 4
+    n_pool = max(1, min(4, int(24e9 // pair_bytes)))
+    pool = [W.gaussian_pair_torch(layout, K, DATA_SEED + 1 + 1000 * r + rank, dev) for r in range(n_pool)]
+    h = binding.Handle(K, P, segs)
+    h.ah_state_set(binding.AH_CENTER, W.theta0_torch(layout, DATA_SEED + rank, dev))
+    h.ah_broadcast_center()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(args.warmup):
+        t = run_period(h, pool, t, wl)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = h.ah_launch_count()
+    events = []
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        t = run_period(h, pool, t, wl, events)
+    stop.record()
+    barrier()
+    ms = start.elapsed_time(stop)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = h.ah_launch_count() - launches0
+    if dist is not None:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    updates = K * P * tau * args.steps * world
+    value = updates / (ms * 1e-3) / 1e9
+
+    # per-launch duration of the fused local-step kernel (plain rounds; the rounds that
+    # also measure distances are listed beside it)
+    plain = [(a.elapsed_time(b), n) for a, b, ex, n in events if not ex]
+    withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex]
+    dom, extra_bytes, dom_name = (plain, 0, "local_step") if plain else (withd, 4 * P, "local_step+dist")
+    dom_ms = sum(d for d, _ in dom) / len(dom)
+    dom_bytes = sum(32 * P * n + extra_bytes for _, n in dom) / len(dom)
+    peak, peak_kind = measured_hbm_peak()
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["sources_sha256"] == kernel_sources_hash() and NCU_TRAFFIC["dram_bytes_per_update"]:
+        traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": traffic,
+                "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
+                "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
+    # whole-period bytes: 32 per update + (8 K_act P + 12 P) per exchange
+    period_bytes = 32 * K * P * tau + 8 * K * P + 12 * P
+    whole = {"algorithmic_GBps": round(period_bytes * args.steps / (ms * 1e-3) / 1e9, 1)}
+    whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
+
+    # end-to-end leg: same periods, inputs copied from pinned host memory every round,
+    # the distances/weights read back every period
+    e2e = None
+    if not args.no_e2e:
+        n_host = 1 if pair_bytes > 4e9 else 2
+        host_pool = [(g.cpu().pin_memory(), hv.cpu().pin_memory()) for g, hv in pool[:n_host]]
+        sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
+        e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
+        t = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+        barrier()
+        start.record()
+        for _ in range(e2e_steps):
+            t = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+        stop.record()
+        barrier()
+        ems = start.elapsed_time(stop)
+        if dist is not None:
+            tmax = torch.tensor([ems], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            ems = float(tmax.item())
+        e2e = {"value": round(K * P * tau * e2e_steps * world / (ems * 1e-3) / 1e9, 3),
+               "unit": "G param-updates/s", "steps": e2e_steps,
+               "h2d_bytes_per_step": pair_bytes * tau, "d2h_bytes_per_step": 8 * K}
+
+    out = {
+        "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
+        "value": round(value, 3), "unit": "G param-updates/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "impl": "cuda",
+        "config": {"workload": f"{args.workload}: {kind} layout, P={P}, K={K}, tau={tau}, "
+                               f"p_fail={p_fail}, max_stale={max_stale}, frozen_stragglers={frozen}",
+                   "step": f"one communication period = {tau} rounds + 1 exchange",
+                   "rounds_timed": tau * args.steps, "input_pool": n_pool,
+                   "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
+                         % ((32 * K * P) / 1e9) if 32 * K * P > 4 * 126e6 else
+                         "working set comparable to L2: partly L2-resident, reported as is",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "roofline": roofline, "whole_step": whole, "e2e": e2e, "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    h.close()
+    del pool
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(args, budget_s=12.0)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def oracle_sample(args, max_params):
+    """The bounded sample of the workload the oracle is timed on: the same K, tau,
+    failure model and hyper-parameters, on the leading whole tensors of the layout up
+    to about max_params parameters (all of it when it is smaller)."""
+    from paper_2409_09242_b200 import workloads as W
+    kind, K, tau, p_fail, max_stale, frozen = WORKLOADS[args.workload]
+    layout = make_layout(kind)
+    keep = []
+    for tns in layout:
+        if keep and tns.offset + tns.numel > max_params:
+            break
+        keep.append(tns)
+    if len(keep) == 1 and keep[0].numel > max_params and len(keep[0].shape) == 1:
+        keep = W.single_segment_layout(max_params)
+    return keep, f"first {len(keep)} of {len(layout)} tensors, P={W.total_params(keep)} of {W.total_params(layout)}"
+
+
+def oracle_periods(args, layout, periods, warm):
+    """Runs warm + periods communication periods of the oracle; returns (seconds, K, P, tau, threads)."""
+    import numpy as np
+    from paper_2409_09242_b200 import workloads as W
+    kind, K, tau, p_fail, max_stale, frozen = WORKLOADS[args.workload]
+    threads = max(1, min(K, len(os.sched_getaffinity(0))))
+    os.environ["OMP_NUM_THREADS"] = str(threads)
+    import oracle
+    segs, P = W.segments(layout), W.total_params(layout)
+    pool = W.gaussian_pool_np(layout, K, 2, DATA_SEED + 1)
+    st = oracle.OracleState(W.theta0_np(layout, DATA_SEED), K, segs, variant="omp")
+    alpha = alpha_for(K)
+    t, t_start = 0, None
+    for period in range(warm + periods):
+        if period == warm:
+            t_start = time.perf_counter()
+        for r in range(tau):
+            t += 1
+            mask = st.mask_next(MASK_SEED, t, p_fail, max_stale)
+            ex = r == tau - 1
+            g, hv = pool[t % 2]
+            st.local_step(g, hv, Z_SEED, t, active=mask if frozen else None, want_dist=ex, **HYPER)
+            if ex:
+                h2, h1 = st.weights_next(alpha)
+                st.exchange(mask, h2, h1)
+    return time.perf_counter() - t_start, K, P, tau, min(threads, st.o.num_threads())
+
+
+def cpu_baseline(args, budget_s):
+    """The CPU oracle, as it stands, timed on this host on a bounded sample."""
+    layout, what = oracle_sample(args, max_params=4_000_000)
+    sec, K, P, tau, threads = oracle_periods(args, layout, periods=1, warm=0)
+    periods = max(1, min(20, int(budget_s / max(sec, 1e-3))))
+    sec, K, P, tau, threads = oracle_periods(args, layout, periods=periods, warm=1)
+    return {"value": round(K * P * tau * periods / sec / 1e9, 5), "unit": "G param-updates/s",
+            "cores": threads, "kind": "oracle",
+            "sample": f"{what}; {periods} periods of {tau} rounds, {sec:.1f} s; OpenMP build, "
+                      f"local steps parallel over workers ({threads} threads)"}
+
+
+def reference_arm(args):
+    """--impl reference: the oracle on the host cores, same metric and config."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    layout, what = oracle_sample(args, max_params=1_000_000)
+    sec, K, P, tau, threads = oracle_periods(args, layout, periods=args.steps, warm=args.warmup)
+    value = round(K * P * tau * args.steps / sec / 1e9, 5)
+    kind = WORKLOADS[args.workload][0]
+    print(json.dumps({
+        "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
+        "value": value, "unit": "G param-updates/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(sec / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "impl": "reference",
+        "config": {"workload": f"{args.workload}: {kind} layout, K={K}, tau={tau} ({what})",
+                   "step": f"one communication period = {tau} rounds + 1 exchange"},
+        "cpu_baseline": {"value": value, "unit": "G param-updates/s", "cores": threads,
+                         "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": "G param-updates/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        gpu_arm(args)
+
+
+if __name__ == "__main__":
+    main()

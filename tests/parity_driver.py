@@ -1,0 +1,99 @@
+"""Drives the CUDA library and the CPU oracle through the same rounds on the same
+seeded inputs, for the parity tests.  Holds no arithmetic of the method itself."""
+from dataclasses import dataclass, field
+
+import numpy as np
+
+Z_SEED = 0x5EED0001
+MASK_SEED = 0x5EED0002
+
+
+@dataclass
+class RunConfig:
+    K: int
+    segments: list
+    P: int
+    rounds: int
+    tau: int
+    p_fail: float = 0.0
+    max_stale: int = 1
+    frozen: bool = False            # a worker that is down also skips its local steps
+    lr: float = 0.01
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-4
+    hessian_power: float = 1.0
+    weight_decay: float = 0.0
+    alpha: float | None = None      # None: min(0.05, 0.8 / K)
+    dynamic: bool = True            # dynamic weights (else fixed alpha)
+    scripted: list = field(default_factory=list)
+    pool: int = 3
+    data_seed: int = 0
+
+    def alpha_value(self):
+        return min(0.05, 0.8 / self.K) if self.alpha is None else self.alpha
+
+
+def tolerance_violations(got, want):
+    """Count of elements outside |got - want| <= 1e-6 + 1e-5 |want| (the parity bar)."""
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    return int(np.count_nonzero(np.abs(got - want) > 1e-6 + 1e-5 * np.abs(want)))
+
+
+def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="omp", check_every=0):
+    """Gaussian grad/hvp pool (configs shaped like the CNN layouts).  layout_inputs =
+    (theta0, [(grad, hvp), ...]) as numpy arrays.  Returns (handle, oracle_state, log)."""
+    import torch
+    from paper_2409_09242_b200 import workloads as W
+
+    theta0, pool = layout_inputs
+    dev_pool = [(torch.from_numpy(g).cuda(), torch.from_numpy(h).cuda()) for g, h in pool]
+    h = binding.Handle(cfg.K, cfg.P, cfg.segments)
+    h.ah_state_set(binding.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    ref = oracle_mod.OracleState(theta0, cfg.K, cfg.segments, variant=variant)
+    alpha = cfg.alpha_value()
+    log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "exchanges": 0}
+    for t in range(1, cfg.rounds + 1):
+        mask_g = h.dw_mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
+        mask_o = ref.mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
+        mask_g = W.apply_scripted(mask_g, t, cfg.scripted)
+        mask_o = W.apply_scripted(mask_o, t, cfg.scripted)
+        log["masks_equal"] &= bool(np.array_equal(mask_g, mask_o))
+        ex = t % cfg.tau == 0
+        k = t % len(pool)
+        common = dict(lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
+                      hessian_power=cfg.hessian_power, weight_decay=cfg.weight_decay,
+                      want_dist=ex)
+        h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
+                        active=mask_g if cfg.frozen else None, **common)
+        ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
+                       active=mask_o if cfg.frozen else None, **common)
+        if ex:
+            log["exchanges"] += 1
+            if cfg.dynamic:
+                w = h.dw_weights_next(alpha)
+                h2, h1 = ref.weights_next(alpha)
+                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+                log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], h2) and
+                                             np.array_equal(w[cfg.K:], h1))
+                h.easgd_exchange(mask_g, w, alpha)
+                ref.exchange(mask_o, h2, h1)
+            else:
+                h.easgd_exchange(mask_g, None, alpha)
+                ref.exchange(mask_o, alpha=alpha)
+        if check_every and t % check_every == 0:
+            assert tolerance_violations(h.ah_state_get(binding.AH_X), ref.x) == 0, t
+    return h, ref, log
+
+
+def compare_state(h, ref, binding):
+    """(violations of the parity bar, count of bit differences) over x, m, v, center."""
+    viol, bits = {}, {}
+    for name, which, want in (("x", binding.AH_X, ref.x), ("m", binding.AH_M, ref.m),
+                              ("v", binding.AH_V, ref.v), ("center", binding.AH_CENTER, ref.center)):
+        got = h.ah_state_get(which)
+        viol[name] = tolerance_violations(got, want)
+        bits[name] = int(np.count_nonzero(got.view(np.uint32) != want.view(np.uint32)))
+    return viol, bits

@@ -1,0 +1,338 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the CPU oracle
+element by element on the same seeded inputs.  Bar: z, masks, weights bit-exact;
+binary32 state within |gpu - oracle| <= 1e-6 + 1e-5 |oracle| (and, because the kernels
+follow the oracle's operation order, in fact bit-identical for hessian power 1 and 1/2)."""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import OracleState
+from paper_2409_09242_b200 import workloads as W
+from parity_driver import RunConfig, compare_state, run_gaussian, tolerance_violations, Z_SEED
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2409_09242_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    torch.cuda.set_device(0)
+    return torch
+
+
+ODD_SEGS = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 256)]
+ODD_P = 13_111
+
+
+def _inputs(segs, P, K, n_pool, seed, scale=0.1):
+    rng = np.random.default_rng(seed)
+    ld = W.padded_ld(P)
+    theta0 = (rng.standard_normal(P) * scale).astype(np.float32)
+    pool = []
+    for _ in range(n_pool):
+        g = np.zeros((K, ld), np.float32)
+        h = np.zeros((K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(scale)
+        h[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(scale)
+        pool.append((g, h))
+    return theta0, pool
+
+
+# ------------------------------------------------------------------------- z
+@pytest.mark.parametrize("K,P", [(4, 1 << 20), (3, 184_837), (2, 129), (1, 1), (5, 4097)])
+def test_sample_z_bit_exact(B, torch, K, P):
+    h = B.Handle(K, P, [])
+    ld = W.padded_ld(P) + 8
+    for seed, t in ((Z_SEED, 1), (0xDEADBEEFCAFEF00D, 77), (0, 0xFFFFFFFE)):
+        dst = torch.full((K, ld), 7.0, dtype=torch.float32, device="cuda")
+        h.ah_sample_z(seed, t, dst)
+        got = dst.cpu().numpy()
+        want = oracle.load("omp").sample_zbits(seed, t, K, P)
+        assert np.array_equal(got[:, :P], np.where(want == 1, -1.0, 1.0).astype(np.float32))
+        assert np.all(got[:, P:] == 7.0)                 # nothing written past P
+    h.close()
+
+
+# ---------------------------------------------------------------- local step
+@pytest.mark.parametrize("segs,P", [
+    ([(0, 5000, 1)], 5000),                      # one unstructured tensor
+    ([], 2048 * 3),                              # no table at all, exact tiles
+    ([(0, 9 * 700, 9)], 6300),                   # blocks straddle tile edges
+    (ODD_SEGS, ODD_P),                           # odd offsets, gaps, block 49/5/256
+    ([(0, 1, 1)], 1), ([(0, 3, 3)], 3), ([(1, 4, 2)], 6),
+])
+@pytest.mark.parametrize("hp,wd", [(1.0, 0.0), (0.5, 0.01), (0.75, 0.0)])
+def test_local_step_matches_oracle(B, torch, segs, P, hp, wd):
+    K, R = 3, 4
+    theta0, pool = _inputs(segs, P, K, 2, seed=P)
+    cfg = RunConfig(K=K, segments=segs, P=P, rounds=R, tau=10 ** 6, lr=0.02, hessian_power=hp,
+                    weight_decay=wd)
+    h, ref, _ = run_gaussian(cfg, B, oracle, (theta0, pool), variant="fp32")
+    viol, bits = compare_state(h, ref, B)
+    assert sum(viol.values()) == 0, viol
+    if hp in (1.0, 0.5):
+        assert sum(bits.values()) == 0, bits           # same operation order => same bits
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    h.close()
+
+
+def test_local_step_inactive_padding_and_auto_round(B, torch):
+    segs, P, K = ODD_SEGS, ODD_P, 4
+    theta0, pool = _inputs(segs, P, K, 1, seed=5)
+    g = torch.from_numpy(pool[0][0]).cuda()
+    hv = torch.from_numpy(pool[0][1]).cuda()
+    # a wider row stride than P, with poison in the padding columns
+    ld = W.padded_ld(P) + 64
+    gw = torch.full((K, ld), float("nan"), device="cuda")
+    hw = torch.full((K, ld), float("nan"), device="cuda")
+    gw[:, :P] = g[:, :P]
+    hw[:, :P] = hv[:, :P]
+    h = B.Handle(K, P, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    ref = OracleState(theta0, K, segs)
+    active = np.array([1, 0, 1, 1], np.uint8)
+    for t in (1, 2, 3):
+        act = active if t == 2 else None
+        h.ah_local_step(gw, hw, Z_SEED, lr=0.01, active=act)          # round = call count
+        ref.local_step(pool[0][0], pool[0][1], Z_SEED, t, lr=0.01, active=act)
+    viol, bits = compare_state(h, ref, B)
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), np.array([3, 2, 3, 3], np.uint32))
+    assert np.array_equal(h.ah_state_get(B.AH_ROUND), np.array([3, 0], np.uint32))
+    h.close()
+
+
+# ------------------------------------------------------------------ distances
+@pytest.mark.parametrize("K,P", [(2, 1), (3, 5), (4, 2048), (2, 2049), (3, 300_001), (1, 1 << 20)])
+def test_norm2_bit_exact(B, torch, K, P):
+    rng = np.random.default_rng(P)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    x = (theta0[None] + rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.01))
+    h = B.Handle(K, P, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x)
+    # a step in which nobody is active leaves x alone and still measures every distance
+    z = torch.zeros((K, W.padded_ld(P)), device="cuda")
+    h.ah_local_step(z, z, 1, lr=0.0, active=np.zeros(K, np.uint8), want_dist=True)
+    got = h.ah_state_get(B.AH_NORM2)
+    want = oracle.load("omp").norm2(np.ascontiguousarray(x), theta0)
+    assert np.array_equal(got, want)
+    assert np.array_equal(h.ah_state_get(B.AH_X), x)
+    h.close()
+
+
+# ------------------------------------------------------------------- exchange
+@pytest.mark.parametrize("K,P", [(1, 7), (3, 1000), (4, 4099), (7, 2048), (16, 10_001), (64, 3001)])
+def test_exchange_bit_exact(B, torch, K, P):
+    rng = np.random.default_rng(K * 1000 + P)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    x = theta0[None] + rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.05)
+    h = B.Handle(K, P, [])
+    ref = OracleState(theta0, K, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x)
+    ref.x[:] = x
+    for trial in range(4):
+        mask = (rng.random(K) > 0.3).astype(np.uint8) if trial else None
+        if trial == 3:
+            mask[:] = 0                                    # nobody reaches the master
+        if trial % 2 == 0:
+            h2 = rng.uniform(0, 0.05, K).astype(np.float32)
+            h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+            h.easgd_exchange(mask, np.concatenate([h2, h1]), 0.0)
+            ref.exchange(mask, h2, h1)
+        else:
+            h.easgd_exchange(mask, None, 0.8 / K)
+            ref.exchange(mask, alpha=0.8 / K)
+        assert np.array_equal(h.ah_state_get(B.AH_X), ref.x), trial
+        assert np.array_equal(h.ah_state_get(B.AH_CENTER), ref.center), trial
+    h.close()
+
+
+def test_exchange_alpha_zero_is_identity(B, torch):
+    K, P = 4, 5000
+    rng = np.random.default_rng(1)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    x = rng.standard_normal((K, P)).astype(np.float32)
+    h = B.Handle(K, P, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x)
+    h.easgd_exchange(None, None, 0.0)
+    assert np.array_equal(h.ah_state_get(B.AH_X), x)
+    assert np.array_equal(h.ah_state_get(B.AH_CENTER), theta0)
+    h.close()
+
+
+# ---------------------------------------------------- whole configurations
+def _check_run(B, cfg, inputs, bit_exact=True):
+    h, ref, log = run_gaussian(cfg, B, oracle, inputs, variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"], log
+    assert sum(viol.values()) == 0, viol
+    if bit_exact:
+        assert sum(bits.values()) == 0, bits
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert log["exchanges"] == cfg.rounds // cfg.tau
+    h.close()
+
+
+def _layout_inputs(layout, K, n_pool=3, seed=0):
+    return W.theta0_np(layout, seed), W.gaussian_pool_np(layout, K, n_pool, seed + 1)
+
+
+def test_config_resnet18_shape_reduced(B, torch):
+    # ResNet-18-shaped layout at 1/8 width (62 tensors, ragged tail), K=8, tau=4,
+    # Bernoulli(0.1) communication failures, 200 rounds
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=200, tau=4,
+                    p_fail=0.1)
+    _check_run(B, cfg, _layout_inputs(layout, 8))
+
+
+@pytest.mark.parametrize("tau", [1, 4, 16])
+def test_config_resnet50_shape_reduced_stragglers(B, torch, tau):
+    # ResNet-50-shaped layout at 1/8 width (161 tensors), K=16, failure 0.2 with
+    # stragglers frozen for 1..8 rounds, 100 rounds per tau
+    layout = W.resnet50_layout(8)
+    cfg = RunConfig(K=16, segments=W.segments(layout), P=W.total_params(layout), rounds=100,
+                    tau=tau, p_fail=0.2, max_stale=8, frozen=True)
+    _check_run(B, cfg, _layout_inputs(layout, 16))
+
+
+def test_config_vgg16_shape_reduced(B, torch):
+    # VGG-16-shaped layout at 1/8 width (long dense tensors), K=4, tau=8, failure 0.25
+    layout = W.vgg16_layout(8)
+    cfg = RunConfig(K=4, segments=W.segments(layout), P=W.total_params(layout), rounds=50, tau=8,
+                    p_fail=0.25)
+    _check_run(B, cfg, _layout_inputs(layout, 4))
+
+
+@pytest.mark.parametrize("K,p_fail", [(4, 0.0), (16, 0.1), (32, 0.3), (64, 0.1)])
+def test_config_worker_sweep_reduced(B, torch, K, p_fail):
+    layout = W.resnet50_layout(16)
+    cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=50, tau=4,
+                    p_fail=p_fail)
+    _check_run(B, cfg, _layout_inputs(layout, K, n_pool=2))
+
+
+def test_config_diagonal_quadratic_full_size(B, torch):
+    """f = 1/2 sum h theta^2, P = 2^20 in one tensor, K = 4, 100 rounds, tau = 4, worker 3
+    cut off from the master in rounds 20..40; exact Hessian-vector products h * z with
+    the z each side samples itself; gradients formed from each side's own x."""
+    K, P, R, tau, alpha, lr = 4, 1 << 20, 100, 4, 0.05, 0.1
+    hq, theta0 = W.quadratic_problem_np(P, 0)
+    outages = [W.scripted_down(3, 20, 40)]
+    segs = W.segments(W.single_segment_layout(P))
+    h = B.Handle(K, P, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    ref = OracleState(theta0, K, segs, variant="omp")
+    orc = oracle.load("omp")
+    hq_dev = torch.from_numpy(hq).cuda()
+    z_dev = torch.empty((K, P), device="cuda")
+    masks_equal = weights_equal = True
+    for t in range(1, R + 1):
+        noise = W.quadratic_noise_np(K, P, 0, t)
+        mask_g = W.apply_scripted(h.dw_mask_next(2, t, 0.0), t, outages)
+        mask_o = W.apply_scripted(ref.mask_next(2, t, 0.0), t, outages)
+        masks_equal &= bool(np.array_equal(mask_g, mask_o))
+        ex = t % tau == 0
+        # device side: its own x, its own z
+        g_dev = torch.from_numpy(W.quadratic_grad_np(hq, h.ah_state_get(B.AH_X), noise)).cuda()
+        h.ah_sample_z(Z_SEED, t, z_dev)
+        hv_dev = hq_dev[None, :] * z_dev
+        h.ah_local_step(g_dev, hv_dev, Z_SEED, lr=lr, round_=t, want_dist=ex)
+        # oracle side
+        g = W.quadratic_grad_np(hq, ref.x, noise)
+        hv = W.quadratic_hvp_np(hq, orc.sample_z(Z_SEED, t, K, P))
+        ref.local_step(g, hv, Z_SEED, t, lr=lr, want_dist=ex)
+        if ex:
+            w = h.dw_weights_next(alpha)
+            h2, h1 = ref.weights_next(alpha)
+            weights_equal &= bool(np.array_equal(w[:K], h2) and np.array_equal(w[K:], h1))
+            h.easgd_exchange(mask_g, w, alpha)
+            ref.exchange(mask_o, h2, h1)
+    assert masks_equal and weights_equal
+    viol, bits = compare_state(h, ref, B)
+    assert sum(viol.values()) == 0, viol
+    assert sum(bits.values()) == 0, bits
+    # Hutchinson is exact on a diagonal Hessian: v is an EMA of h^2 alone, noise-free
+    v = h.ah_state_get(B.AH_V)
+    bc2 = 1.0 - float(np.float32(0.999)) ** R
+    assert np.allclose(v[0] / bc2, hq.astype(np.float64) ** 2, rtol=1e-4)
+    h.close()
+
+
+# ------------------------------------------------ checkpoint / resume, errors
+def test_checkpoint_resume_is_bit_identical(B, torch):
+    layout = W.resnet18_layout(16)
+    segs, P, K = W.segments(layout), W.total_params(layout), 4
+    inputs = _layout_inputs(layout, K)
+    full = RunConfig(K=K, segments=segs, P=P, rounds=24, tau=4, p_fail=0.2, max_stale=4, frozen=True)
+    half = RunConfig(K=K, segments=segs, P=P, rounds=12, tau=4, p_fail=0.2, max_stale=4, frozen=True)
+    h_full, _, _ = run_gaussian(full, B, oracle, inputs, variant="omp")
+    h_a, ref_a, _ = run_gaussian(half, B, oracle, inputs, variant="omp")
+    # snapshot, restore into a fresh handle, continue rounds 13..24 by hand
+    snap = {w: h_a.ah_state_get(w) for w in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER, B.AH_STEP,
+                                             B.AH_UHIST, B.AH_DOWN_UNTIL, B.AH_ROUND)}
+    h_a.close()
+    h_b = B.Handle(K, P, segs)
+    for w, val in snap.items():
+        h_b.ah_state_set(w, val)
+    dev_pool = [(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda()) for g, hv in inputs[1]]
+    from parity_driver import MASK_SEED
+    alpha = full.alpha_value()
+    for t in range(13, 25):
+        mask = h_b.dw_mask_next(MASK_SEED, t, 0.2, 4)
+        ex = t % 4 == 0
+        g, hv = dev_pool[t % len(dev_pool)]
+        h_b.ah_local_step(g, hv, Z_SEED, lr=0.01, round_=t, active=mask, want_dist=ex)
+        if ex:
+            h_b.easgd_exchange(mask, h_b.dw_weights_next(alpha), alpha)
+    for w in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER):
+        a, b = h_full.ah_state_get(w), h_b.ah_state_get(w)
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), w
+    assert np.array_equal(h_full.ah_state_get(B.AH_UHIST), h_b.ah_state_get(B.AH_UHIST))
+    h_full.close()
+    h_b.close()
+
+
+def test_error_paths_and_own_allocation(B, torch):
+    K, P = 2, 1000
+    h = B.Handle(K, P, [], own_alloc=True)           # cudaMalloc workspace, default stream
+    g = torch.zeros((K, 1004), device="cuda")
+    lib = B.raw()
+    hy = B.ah_hyper(0.01, 0.9, 0.999, 1e-4, 1.0, 0.0, 1, None, 0)
+    # misaligned base pointer, stride not a multiple of 4, stride below P, null pointer
+    assert lib.ah_local_step(h._h, g.data_ptr() + 4, g.data_ptr(), 1004, 1, C.byref(hy)) == B.AH_ERR_ALIGN
+    assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 1002, 1, C.byref(hy)) == B.AH_ERR_ALIGN
+    assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 996, 1, C.byref(hy)) == B.AH_ERR_INVALID_ARG
+    assert lib.ah_local_step(h._h, None, g.data_ptr(), 1004, 1, C.byref(hy)) == B.AH_ERR_INVALID_ARG
+    bad = B.ah_hyper(0.01, 1.0, 0.999, 1e-4, 1.0, 0.0, 1, None, 0)      # beta1 = 1
+    assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 1004, 1, C.byref(bad)) == B.AH_ERR_INVALID_ARG
+    # weights before any distance has been measured
+    w = (C.c_float * (2 * K))()
+    assert lib.dw_weights_next(h._h, 0.1, w) == B.AH_ERR_STATE
+    assert lib.ah_state_get(h._h, 99, 0, g.data_ptr(), 1) == B.AH_ERR_INVALID_ARG
+    assert lib.ah_state_get(h._h, B.AH_X, K, g.data_ptr(), 1) == B.AH_ERR_INVALID_ARG
+    # the handle still works after the refusals
+    h.ah_local_step(g, g, 1, lr=0.01, want_dist=True)
+    assert np.all(h.dw_weights_next(0.1) == np.float32(0.1))
+    assert h.ah_launch_count() == 2
+    h.close()
+    # a workspace that is too small is refused
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    opt = B.ah_alloc((small.data_ptr() + 255) // 256 * 256, 512, None, 0)
+    out = C.c_void_p(None)
+    assert lib.ah_init(C.byref(out), 4, 10_000, None, 0, C.byref(opt)) == B.AH_ERR_ALLOC
+    assert out.value is None
