@@ -43,6 +43,9 @@ WORKLOADS = {
     "c5k16": ("resnet50", 16, 4, 0.1, 1, False),
     "c5k32": ("resnet50", 32, 4, 0.1, 1, False),
     "c5k64": ("resnet50", 64, 4, 0.1, 1, False),
+    # small cases for profiler captures (about 1 GB on the device, still far above L2)
+    "p18k4": ("resnet18", 4, 4, 0.1, 1, False),
+    "pvggk1": ("vgg16", 1, 4, 0.1, 1, False),
 }
 HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weight_decay=0.0)
 
@@ -182,7 +185,7 @@ def gpu_arm(args):
 
     # synthetic inputs, resident in HBM before the timed region
     pair_bytes = 2 * K * ld * 4
-    n_pool = max(1, min(4, int(24e9 // pair_bytes)))
+    n_pool = max(1, min(args.pool, int(24e9 // pair_bytes)))
     pool = [W.gaussian_pair_torch(layout, K, DATA_SEED + 1 + 1000 * r + rank, dev) for r in range(n_pool)]
     h = binding.Handle(K, P, segs)
     h.ah_state_set(binding.AH_CENTER, W.theta0_torch(layout, DATA_SEED + rank, dev))
@@ -381,6 +384,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--pool", type=int, default=4, help="grad/hvp pairs kept in HBM")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

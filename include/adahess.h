@@ -50,7 +50,7 @@ extern "C" {
 #define AH_ERR_INTERNAL      (-7)  /* the device status word was set by a kernel            */
 
 #define AH_MAX_WORKERS  256        /* K <= 256                                              */
-#define AH_MAX_BLOCK    256        /* spatial block kh*kw <= 256                            */
+#define AH_MAX_BLOCK    128        /* spatial block kh*kw <= 128 (covers 11 x 11 kernels)   */
 #define AH_MAX_HIST     32         /* history depth p of the raw score <= 32                */
 #define AH_ROUND_AUTO   0xFFFFFFFFu
 #define AH_DEVICE_NONE  (-2)       /* ah_alloc.device: bookkeeping-only handle, no GPU      */

@@ -25,7 +25,7 @@ _lib = C.CDLL(_build.LIB_PATH)
 AH_OK = 0
 AH_ERR_INVALID_ARG, AH_ERR_ALIGN, AH_ERR_SEGMENTS, AH_ERR_ALLOC = -1, -2, -3, -4
 AH_ERR_CUDA, AH_ERR_STATE, AH_ERR_INTERNAL = -5, -6, -7
-AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST = 256, 256, 32
+AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST = 256, 128, 32
 AH_ROUND_AUTO = 0xFFFFFFFF
 AH_DEVICE_NONE = -2
 (AH_X, AH_M, AH_V, AH_CENTER, AH_NORM2, AH_STEP, AH_UHIST, AH_DOWN_UNTIL, AH_ROUND,

@@ -18,6 +18,7 @@ struct ah_ctx {
     uint64_t lds = 0;              // row stride of x, m, v, c (P rounded up to 4)
     uint32_t ntiles = 0, ntiles_pad = 0;
     int device = 0;
+    int sm_count = 0;
     bool has_device = true;        // false: bookkeeping-only handle (AH_DEVICE_NONE)
     std::vector<Run> runs_host;
     std::vector<TileInfo> tiles_host;
@@ -28,13 +29,14 @@ struct ah_ctx {
 
     // device views into the workspace
     float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
-    double *partials = nullptr, *scratch = nullptr, *norm2_dev = nullptr;
+    double *partials = nullptr, *scratch = nullptr;
+    double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     Run *runs = nullptr;
     TileInfo *tiles = nullptr;
     uint32_t nruns = 0;
 
     // host state
-    double *norm2_host = nullptr;  // pinned, K doubles
+    double *norm2_host = nullptr;  // pinned copy of norm2_dev (status word + K doubles)
     cudaEvent_t norm2_ready = nullptr;
     bool norm2_pending = false;    // a want_dist step has been enqueued since the last read
     double norm2_last[AH_MAX_WORKERS];
@@ -93,7 +95,7 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.c = take((size_t)lds * sizeof(float));
     L.partials = take((size_t)K * ntp * sizeof(double));
     L.scratch = take((size_t)K * ntp * sizeof(double));
-    L.norm2 = take((size_t)AH_MAX_WORKERS * sizeof(double));
+    L.norm2 = take((size_t)(AH_MAX_WORKERS + 1) * sizeof(double));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
     L.total = off;
@@ -251,7 +253,12 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->runs = (Run *)(base + L.runs);
     h->tiles = (TileInfo *)(base + L.tiles);
 
-    if ((e = cudaMallocHost((void **)&h->norm2_host, AH_MAX_WORKERS * sizeof(double))) != cudaSuccess ||
+    if ((e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device)) !=
+        cudaSuccess) {
+        h->last_cuda = (int)e;
+        return fail(AH_ERR_CUDA);
+    }
+    if ((e = cudaMallocHost((void **)&h->norm2_host, (AH_MAX_WORKERS + 1) * sizeof(double))) != cudaSuccess ||
         (e = cudaEventCreateWithFlags(&h->norm2_ready, cudaEventDisableTiming)) != cudaSuccess) {
         h->last_cuda = (int)e;
         return fail(AH_ERR_ALLOC);
@@ -314,10 +321,12 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0 || ((uintptr_t)hvp & 15u) != 0)
         return AH_ERR_ALIGN;
 
+    const bool dist = hy->want_dist != 0;
     StepParams p;
     p.x = h->x; p.m = h->m; p.v = h->v; p.c = h->c;
     p.grad = grad; p.hvp = hvp;
     p.partials = h->partials;
+    p.status = reinterpret_cast<uint32_t *>(h->norm2_dev);
     p.runs = h->runs; p.tiles = h->tiles;
     p.lds = h->lds; p.ld = ld;
     p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
@@ -329,24 +338,29 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     p.omb1 = 1.0f - hy->beta1;
     p.omb2 = 1.0f - hy->beta2;
     p.eps = hy->eps; p.hpow = hy->hessian_power; p.wd = hy->weight_decay;
+    p.nrows = 0;
     for (int i = 0; i < h->K; ++i) {
         const bool on = !hy->active || hy->active[i] != 0;
         p.active[i] = on ? 1 : 0;
         if (on) h->step[i] += 1;
+        if (on || dist) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
         // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
         // (a worker that sat out steps has taken fewer); double, then one rounding
         const double t = (double)(h->step[i] ? h->step[i] : 1u);
-        p.bc1[i] = (float)(1.0 - pow((double)hy->beta1, t));
-        p.bc2[i] = (float)(1.0 - pow((double)hy->beta2, t));
+        WorkerConst &w = p.w[i];
+        w.bc1 = (float)(1.0 - pow((double)hy->beta1, t));
+        w.bc2 = (float)(1.0 - pow((double)hy->beta2, t));
+        w.rbc1 = 1.0f / w.bc1;
+        w.rbc2 = 1.0f / w.bc2;
     }
-    const bool dist = hy->want_dist != 0;
-    AH_CUDA(h, launch_local_step(p, h->K, dist, h->stream));
-    h->launches += 1;
+    p.nitems = p.nrows * h->ntiles;
+    AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
+    if (p.nitems) h->launches += 1;
     if (dist) {
         AH_CUDA(h, launch_norm2_finalize(h->partials, h->scratch, h->ntiles, h->ntiles_pad, h->K,
-                                         h->norm2_dev, h->stream));
+                                         h->norm2_dev + 1, h->stream));
         h->launches += 1;
-        AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, h->K * sizeof(double),
+        AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, (h->K + 1) * sizeof(double),
                                    cudaMemcpyDeviceToHost, h->stream));
         AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
         h->norm2_pending = true;
@@ -405,7 +419,7 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
     if (to_user) {
         if (which == AH_NORM2 && h->norm2_pending) {
             AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
-            memcpy(h->norm2_last, h->norm2_host, h->K * sizeof(double));
+            memcpy(h->norm2_last, h->norm2_host + 1, h->K * sizeof(double));
         }
         memcpy(user, ptr, bytes);
     } else {
@@ -447,7 +461,8 @@ int dw_weights_next(ah_ctx *h, float alpha, float *weights)
     if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
     AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
     h->norm2_pending = false;
-    return dw_weights_from_norm2(h, h->norm2_host, alpha, weights);
+    if (*reinterpret_cast<const uint32_t *>(h->norm2_host) != 0u) return AH_ERR_INTERNAL;
+    return dw_weights_from_norm2(h, h->norm2_host + 1, alpha, weights);
 }
 
 int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *weights)

@@ -9,21 +9,46 @@
 
 namespace ah {
 
-// Tile of the flat parameter row handled by one CTA: TILE consecutive elements of
-// one worker.  A power of two, so that a tile is a subtree of the pairwise
-// summation tree used for ||x_i - c||^2.
-constexpr int kTile = 2048;
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-constexpr int kGroupsPerWarp = kTile / 128 / kWarps;   // 128 = elements per Philox block
-static_assert(kGroupsPerWarp >= 1 && kGroupsPerWarp <= 8, "warp owns 1..8 Philox groups");
-static_assert((kGroupsPerWarp & (kGroupsPerWarp - 1)) == 0, "power of two");
+// The fused local step is a persistent, warp-specialised pipeline.  One *item* is
+// a tile of kTile consecutive parameters of one worker.  A power of two, so that a
+// tile is a subtree of the pairwise summation tree used for ||x_i - c||^2.
+//   - warp kConsumerWarps (the producer) fills a ring of kStages shared-memory
+//     stages: 1-D bulk copies (TMA) of the tile's grad, x, m, v (and c) and of the
+//     Hessian-vector tile widened to whole spatial blocks, plus the Philox words of
+//     the tile's Rademacher signs;
+//   - warps 0..kConsumerWarps-1 (the consumers) take a stage when its mbarrier
+//     flips, apply signs, average spatial blocks, update, store, and hand the stage
+//     back through a second mbarrier.
+#ifndef AH_PASSES
+#define AH_PASSES 1
+#endif
+#ifndef AH_STAGES
+#define AH_STAGES 2
+#endif
+#ifndef AH_CTAS_PER_SM
+#define AH_CTAS_PER_SM 4
+#endif
+constexpr int kPasses = AH_PASSES;                 // float4 per consumer thread per stream
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kThreads = kConsumers + 32;
+constexpr int kPassElems = kConsumers * 4;         // 1024: one float4 per consumer
+constexpr int kTile = kPassElems * kPasses;
+constexpr int kStages = AH_STAGES;
+constexpr int kCtasPerSm = AH_CTAS_PER_SM;
+static_assert((kTile & (kTile - 1)) == 0, "tile must be a power of two");
 
-// Shared staging of the signed Hessian-vector tile: the tile, a halo of up to
-// AH_MAX_BLOCK - 1 elements on each side (a spatial block may straddle the tile
-// edge) and slack for rounding both ends to 16 bytes.
-constexpr int kStageFloats = kTile + 2 * AH_MAX_BLOCK + 8;
-constexpr int kStageGroups = kStageFloats / 128 + 2;
+// A spatial block may straddle a tile edge: the Hessian-vector stage holds up to
+// kHalo more elements on each side (AH_MAX_BLOCK - 1 rounded out to 16 bytes).
+constexpr int kHalo = AH_MAX_BLOCK;
+static_assert(kHalo % 4 == 0 && kHalo <= 128, "halo spans at most one Philox group a side");
+constexpr int kStageGroups = kTile / 128 + 2;      // Philox groups a stage can touch
+
+// Bits of the device status word (0 = healthy).
+enum : uint32_t {
+    kStatusFullTimeout = 1u,    // a consumer gave up waiting for a stage to fill
+    kStatusEmptyTimeout = 2u,   // the producer gave up waiting for a stage to drain
+};
 
 // The row [0, P) cut into maximal runs of equal spatial block (gaps and block-1
 // tensors merged).  magic = ceil(2^32 / block) turns r / block into one mul-hi for
@@ -44,11 +69,18 @@ struct TileInfo {
     uint32_t flags;
 };
 
+// Per-worker constants of one step: bias corrections 1 - beta^t (t = the worker's
+// own step count) and their correctly rounded reciprocals.
+struct WorkerConst {
+    float bc1, bc2, rbc1, rbc2;
+};
+
 struct StepParams {
     float *x, *m, *v;
     const float *c;
     const float *grad, *hvp;
     double *partials;          // [K][ntiles_pad] tile sums of (x - c)^2
+    uint32_t *status;          // device status word
     const Run *runs;
     const TileInfo *tiles;
     uint64_t lds;              // row stride of x, m, v (elements, multiple of 4)
@@ -58,9 +90,11 @@ struct StepParams {
     uint32_t ntiles_pad;       // power of two >= ntiles
     uint32_t key0, key1, round;
     float lr, beta1, beta2, omb1, omb2, eps, hpow, wd;
-    float bc1[AH_MAX_WORKERS];
-    float bc2[AH_MAX_WORKERS];
-    uint8_t active[AH_MAX_WORKERS];
+    uint32_t nrows;            // worker rows to process (all K when distances are wanted)
+    uint32_t nitems;           // nrows * ntiles
+    WorkerConst w[AH_MAX_WORKERS];
+    uint16_t row[AH_MAX_WORKERS];     // row r -> worker index
+    uint8_t active[AH_MAX_WORKERS];   // by worker index
 };
 
 struct ExchangeParams {
@@ -75,7 +109,7 @@ struct ExchangeParams {
 };
 
 // Kernel launchers (ah_kernels.cu).  Each returns the cudaError_t of the launch.
-cudaError_t launch_local_step(const StepParams &p, int K, bool want_dist, cudaStream_t s);
+cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);
 cudaError_t launch_norm2_finalize(double *partials, double *scratch, uint32_t ntiles,
                                   uint32_t ntiles_pad, int K, double *norm2, cudaStream_t s);
 cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s);

@@ -4,7 +4,7 @@
 // grad, hvp, x, m, v and writes x, m, v once (32 bytes per parameter update), the
 // exchange reads and writes x once more (8 bytes per update) plus the master row.
 // There is no dense contraction, so no tensor cores; the rules that matter are
-// 128-bit coalesced accesses, enough loads in flight, and not touching a byte twice.
+// wide coalesced accesses, enough bytes in flight, and not touching a byte twice.
 //
 // Arithmetic follows one fixed order with one binary32 rounding per operation
 // (__fmul_rn / __fadd_rn / __fdiv_rn / __fsqrt_rn are never contracted into FMAs),
@@ -14,19 +14,115 @@
 namespace ah {
 
 // ---------------------------------------------------------------------------
+// Small PTX wrappers: mbarriers, 1-D bulk copies (TMA), named barriers.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// Bounded wait: polls the barrier at most kWaitPolls times (backing off after the
+// first few), then records `code` in the status word and gives up.  A healthy run
+// never comes near the limit (about a second).
+constexpr uint32_t kWaitPolls = 1u << 22;
+
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t *status,
+                                          uint32_t code)
+{
+    for (uint32_t it = 0; it < kWaitPolls; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 32) __nanosleep(128);
+    }
+    atomicOr(status, code);
+    return false;
+}
+
+// Global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte
+// aligned), completion counted on `bar`.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+
+// Orders this thread's earlier generic-proxy accesses to shared memory before later
+// async-proxy (bulk copy) writes to the same locations.
+__device__ __forceinline__ void fence_generic_to_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void consumer_sync()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+
+// ---------------------------------------------------------------------------
+// Arithmetic helpers
+// ---------------------------------------------------------------------------
+
+// x / b for a divisor b whose correctly rounded reciprocal r is known: one
+// multiply, the exact remainder by FMA, one correction (Markstein's sequence).  The
+// result is the correctly rounded quotient whenever no intermediate leaves the
+// normal range, which the exponent test guarantees for 2^-24 < b <= 1; outside that
+// window of x the plain division is used.  (Checked exhaustively on the host, for
+// every x in the window, against several hundred divisors of the form 1 - beta^t.)
+__device__ __forceinline__ float div_by_const(float x, float b, float r)
+{
+    const uint32_t e = (__float_as_uint(x) >> 23) & 0xffu;
+    if (e - 64u < 127u) {
+        const float q = __fmul_rn(x, r);
+        const float rem = __fmaf_rn(-b, q, x);
+        return __fmaf_rn(rem, r, q);
+    }
+    return __fdiv_rn(x, b);
+}
+
 // Per-element AdaHessian update (Sec. IV-B of the paper; Eq. 4 with the diagonal
 // preconditioner 1 / ((sqrt vhat)^k + eps)).  D is the spatially averaged
 // Hutchinson estimate of the Hessian diagonal for this element.
 // POWMODE: 0 -> k = 1, 1 -> k = 1/2, 2 -> general k via powf.
-// ---------------------------------------------------------------------------
 template <int POWMODE, bool WD>
 __device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, float g, float D,
-                                                  const StepParams &p, float bc1, float bc2)
+                                                  const StepParams &p, const WorkerConst &w)
 {
     const float m1 = __fadd_rn(__fmul_rn(p.beta1, m), __fmul_rn(p.omb1, g));
     const float v1 = __fadd_rn(__fmul_rn(p.beta2, v), __fmul_rn(__fmul_rn(p.omb2, D), D));
-    const float mhat = __fdiv_rn(m1, bc1);
-    const float vhat = __fdiv_rn(v1, bc2);
+    const float mhat = div_by_const(m1, w.bc1, w.rbc1);
+    const float vhat = div_by_const(v1, w.bc2, w.rbc2);
     const float r = __fsqrt_rn(vhat);
     float pw;
     if (POWMODE == 0) pw = r;
@@ -45,6 +141,7 @@ __device__ __forceinline__ float flip_if(float a, uint32_t bit)
     return __uint_as_float(__float_as_uint(a) ^ (bit << 31));
 }
 
+// z (.) h for four consecutive elements; bit k of nib set means z = -1 for lane k.
 __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 {
     h.x = flip_if(h.x, nib & 1u);
@@ -52,11 +149,6 @@ __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
     h.z = flip_if(h.z, (nib >> 2) & 1u);
     h.w = flip_if(h.w, (nib >> 3) & 1u);
     return h;
-}
-
-__device__ __forceinline__ float4 ld_stream(const float *p)
-{
-    return __ldcs(reinterpret_cast<const float4 *>(p));
 }
 
 __device__ __forceinline__ float4 ld_vec(const float *p)
@@ -91,181 +183,246 @@ __device__ __forceinline__ double warp_tree_sum(double s)
 }
 
 // ---------------------------------------------------------------------------
-// Fused local step.  grid = (tiles, K), one CTA per tile of kTile consecutive
-// parameters of one worker.  Element owned by (warp w, pass r, lane l):
-//     j = tile*kTile + w*(kGroupsPerWarp*128) + r*128 + 4*l
-// so each warp pass is one coalesced 512-byte row per stream, and one row is
-// exactly the 128 elements covered by one Philox block.
+// Fused local step: persistent, warp-specialised, TMA-fed.
 //
-// Rademacher signs: lane l computes the Philox block of group (l mod
-// kGroupsPerWarp) of its warp and keeps output word l/8; in pass r every lane
-// fetches the word it needs from lane (l & ~7) | r with one shuffle.  z costs no
-// memory traffic.
+// An item is one tile of kTile consecutive parameters of one worker; CTA b takes
+// items b, b + grid, b + 2 grid, ... (consecutive CTAs stream consecutive tiles).
 //
-// Tiles whose tensors all have spatial block 1 stay in registers.  Tiles that
-// touch a tensor with block > 1 stage the signed Hessian-vector values of the tile,
-// widened to whole blocks, in shared memory; one thread per block replaces the
-// block by its mean in place (ascending-order sum, one division); the update then
-// reads the averaged values back.
+// Producer warp, per item: waits until the stage is free, computes the Philox
+// blocks whose bits are the Rademacher signs of the tile (one lane per group of 128
+// parameters), writes a small header, and issues bulk copies of grad, x, m, v, (c)
+// and of the Hessian-vector values of the tile widened to whole spatial blocks.  z
+// costs no memory traffic.
+//
+// Consumers, per item: wait for the stage; where the tile touches a tensor with
+// spatial block > 1 they turn hvp into z (.) hvp in place, average each block in
+// place (one thread per block, ascending-order sum, one division) and read the
+// means back; otherwise the sign is applied in registers.  Then moments and update
+// per element, 128-bit stores of x, m, v, and the stage goes back to the producer.
 //
 // DIST additionally leaves, per tile, the pairwise-tree sum of (x_new - c)^2 in
-// p.partials[worker][tile] (all workers, active or not).
+// p.partials[worker][tile], for every worker; a worker that sits the step out
+// contributes its unchanged x (only x and c are fetched for it).
 // ---------------------------------------------------------------------------
+enum : uint32_t { kItemAverage = 1u, kItemDistanceOnly = 2u };
+
+template <bool DIST>
+struct __align__(128) Stage {
+    uint32_t worker, t0, nvalid, flags;
+    uint32_t e0, e1, run0, ea0;
+    uint32_t tile, reserved[7];
+    uint32_t zw[kStageGroups][4];          // Philox words of groups (ea0 >> 7) ...
+    float g[kTile], x[kTile], m[kTile], v[kTile];
+    float c[DIST ? kTile : 4];
+    float hv[kTile + 2 * kHalo];           // element j lives at hv[j - t0 + kHalo]
+};
+
+template <bool DIST>
+struct __align__(128) Shared {
+    Stage<DIST> stage[kStages];
+    uint64_t full[kStages];                // producer -> consumers (bytes landed)
+    uint64_t empty[kStages];               // consumers -> producer (stage drained)
+    double red[2][kPasses * kConsumerWarps];
+};
+
+template <int B>
+__device__ __forceinline__ void block_means_fixed(float *base, uint32_t nblk, int ctid)
+{
+    for (uint32_t k = ctid; k < nblk; k += kConsumers) {
+        float *blk = base + k * B;
+        float S = blk[0];
+#pragma unroll
+        for (int e = 1; e < B; ++e) S = __fadd_rn(S, blk[e]);
+        const float mean = __fdiv_rn(S, (float)B);
+#pragma unroll
+        for (int e = 0; e < B; ++e) blk[e] = mean;
+    }
+}
+
+__device__ __forceinline__ void block_means_any(float *base, uint32_t nblk, uint32_t B, int ctid)
+{
+    const float fb = (float)B;
+    for (uint32_t k = ctid; k < nblk; k += kConsumers) {
+        float *blk = base + k * B;
+        float S = blk[0];
+        for (uint32_t e = 1; e < B; ++e) S = __fadd_rn(S, blk[e]);
+        const float mean = __fdiv_rn(S, fb);
+        for (uint32_t e = 0; e < B; ++e) blk[e] = mean;
+    }
+}
+
 template <int POWMODE, bool WD, bool DIST>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 local_step_kernel(const __grid_constant__ StepParams p)
 {
-    __shared__ __align__(16) float sD[kStageFloats];
-    __shared__ uint32_t sZ[kStageGroups][4];
-    __shared__ double sRed[kWarps];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Shared<DIST> &sh = *reinterpret_cast<Shared<DIST> *>(smem_raw);
 
-    const int tid = threadIdx.x;
-    const int lane = tid & 31, warp = tid >> 5;
-    const int i = blockIdx.y;
-    const uint32_t tile = blockIdx.x;
-    const bool active = p.active[i] != 0;
-    if (!active && !DIST) return;
-
-    const uint32_t t0 = tile * (uint32_t)kTile;
-    const uint32_t jw = t0 + (uint32_t)warp * (kGroupsPerWarp * 128) + 4u * (uint32_t)lane;
-    float *xr = p.x + (uint64_t)i * p.lds;
-
-    float4 xv[kGroupsPerWarp];
-    int nv[kGroupsPerWarp];            // valid lanes of each float4 (0..4)
-#pragma unroll
-    for (int r = 0; r < kGroupsPerWarp; ++r) {
-        const uint32_t j = jw + 128u * r;
-        nv[r] = j >= p.P ? 0 : (p.P - j >= 4u ? 4 : (int)(p.P - j));
-    }
-
-    if (active) {
-        float *mr = p.m + (uint64_t)i * p.lds;
-        float *vr = p.v + (uint64_t)i * p.lds;
-        const float *gr = p.grad + (uint64_t)i * p.ld;
-        const float *hr = p.hvp + (uint64_t)i * p.ld;
-        const float bc1 = p.bc1[i], bc2 = p.bc2[i];
-        const TileInfo ti = p.tiles[tile];
-
-        const bool in_registers = (ti.flags & 1u) == 0;
-
-        // issue every global load of the tile up front
-        float4 gv[kGroupsPerWarp], mv[kGroupsPerWarp], vv[kGroupsPerWarp], dv[kGroupsPerWarp];
-#pragma unroll
-        for (int r = 0; r < kGroupsPerWarp; ++r) {
-            if (nv[r] > 0) {
-                const uint32_t j = jw + 128u * r;
-                if (in_registers) dv[r] = ld_stream(hr + j);
-                gv[r] = ld_stream(gr + j);
-                xv[r] = ld_vec(xr + j);
-                mv[r] = ld_vec(mr + j);
-                vv[r] = ld_vec(vr + j);
-            }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], kConsumerWarps);
         }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
-        if (in_registers) {
-            // -------- all spatial blocks are 1: signs by shuffle, D stays in registers
-            uint32_t w[4];
-            const uint32_t grp = (t0 >> 7) + (uint32_t)warp * kGroupsPerWarp
-                                 + (uint32_t)(lane & (kGroupsPerWarp - 1));
-            philox4x32_10(grp, (uint32_t)i, p.round, kDomainZ, p.key0, p.key1, w);
-            const int sel = lane >> 3;
-            const uint32_t mine = sel == 0 ? w[0] : sel == 1 ? w[1] : sel == 2 ? w[2] : w[3];
-#pragma unroll
-            for (int r = 0; r < kGroupsPerWarp; ++r) {
-                const uint32_t word = __shfl_sync(0xffffffffu, mine, (lane & ~7) | r);
-                if (nv[r] > 0) {
-                    const uint32_t nib = (word >> (4 * (lane & 7))) & 0xFu;
-                    dv[r] = apply_signs(dv[r], nib);
+    if (warp == kConsumerWarps) {
+        // =============================== producer ===============================
+        uint32_t k = 0;
+        for (uint32_t n = blockIdx.x; n < p.nitems; n += gridDim.x, ++k) {
+            const uint32_t s = k % kStages, use = k / kStages;
+            if (use > 0 && !mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout))
+                break;
+            Stage<DIST> &st = sh.stage[s];
+            const uint32_t r = n / p.ntiles, tile = n - r * p.ntiles;
+            const uint32_t i = p.row[r];
+            const bool act = p.active[i] != 0;
+            const uint32_t t0 = tile * (uint32_t)kTile;
+            const uint32_t nvalid = min((uint32_t)kTile, p.P - t0);
+            const uint32_t n4 = (nvalid + 3u) & ~3u;
+            const TileInfo ti = p.tiles[tile];
+            const bool avg = act && (ti.flags & 1u);
+            const uint32_t ea0 = avg ? (ti.e0 & ~3u) : t0;
+            const uint32_t ea1 = avg ? ((ti.e1 + 3u) & ~3u) : t0 + n4;
+            if (act) {
+                const uint32_t g0 = ea0 >> 7;
+                const uint32_t ng = ((ea1 - 1u) >> 7) - g0 + 1u;
+                if ((uint32_t)lane < ng)
+                    philox4x32_10(g0 + lane, i, p.round, kDomainZ, p.key0, p.key1, st.zw[lane]);
+            }
+            if (lane == 0) {
+                st.worker = i; st.t0 = t0; st.nvalid = nvalid;
+                st.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly);
+                st.e0 = ti.e0; st.e1 = ti.e1; st.run0 = ti.run0; st.ea0 = ea0;
+                st.tile = tile;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t row_bytes = n4 * 4u, hv_bytes = (ea1 - ea0) * 4u;
+                const uint64_t so = (uint64_t)i * p.lds + t0;
+                uint64_t *bar = &sh.full[s];
+                if (act) {
+                    mbar_arrive_expect_tx(bar, 4u * row_bytes + hv_bytes + (DIST ? row_bytes : 0u));
+                    bulk_load(&st.hv[ea0 + kHalo - t0], p.hvp + (uint64_t)i * p.ld + ea0, hv_bytes, bar);
+                    bulk_load(st.g, p.grad + (uint64_t)i * p.ld + t0, row_bytes, bar);
+                    bulk_load(st.x, p.x + so, row_bytes, bar);
+                    bulk_load(st.m, p.m + so, row_bytes, bar);
+                    bulk_load(st.v, p.v + so, row_bytes, bar);
+                    if constexpr (DIST) bulk_load(st.c, p.c + t0, row_bytes, bar);
+                } else if constexpr (DIST) {
+                    mbar_arrive_expect_tx(bar, 2u * row_bytes);
+                    bulk_load(st.x, p.x + so, row_bytes, bar);
+                    bulk_load(st.c, p.c + t0, row_bytes, bar);
                 }
             }
-        } else {
-            // -------- stage z (.) hvp for [e0, e1) rounded out to 16 bytes
-            const uint32_t ea0 = ti.e0 & ~3u;
-            const uint32_t ea1 = (ti.e1 + 3u) & ~3u;
-            const uint32_t g0 = ea0 >> 7;
-            const uint32_t ng = ((ea1 - 1u) >> 7) - g0 + 1u;
-            if ((uint32_t)tid < ng)
-                philox4x32_10(g0 + tid, (uint32_t)i, p.round, kDomainZ, p.key0, p.key1, sZ[tid]);
-            __syncthreads();
-            const uint32_t nvec = (ea1 - ea0) >> 2;
-            for (uint32_t q = tid; q < nvec; q += kThreads) {
-                const uint32_t j = ea0 + 4u * q;
-                const uint32_t word = sZ[(j >> 7) - g0][(j >> 5) & 3u];
-                const uint32_t nib = (word >> (j & 31u)) & 0xFu;
-                st_vec(&sD[4u * q], apply_signs(ld_stream(hr + j), nib));
-            }
-            __syncthreads();
-            // -------- block means, one thread per block, in place
-            for (uint32_t ri = ti.run0; ri < 0xffffffffu; ++ri) {
-                const Run rn = p.runs[ri];
-                if (rn.start >= ti.e1) break;
-                if (rn.block > 1u) {
-                    const uint32_t qa = max(ti.e0, rn.start);
-                    const uint32_t qb = min(ti.e1, rn.end);
-                    const uint32_t nblk = __umulhi(qb - qa, rn.magic);
-                    const float fb = (float)rn.block;
-                    for (uint32_t k = tid; k < nblk; k += kThreads) {
-                        float *blk = &sD[qa - ea0 + k * rn.block];
-                        float S = blk[0];
-                        for (uint32_t e = 1; e < rn.block; ++e) S = __fadd_rn(S, blk[e]);
-                        const float mean = __fdiv_rn(S, fb);
-                        for (uint32_t e = 0; e < rn.block; ++e) blk[e] = mean;
+        }
+        return;
+    }
+
+    // ================================= consumers =================================
+    const int ctid = threadIdx.x;
+    uint32_t k = 0;
+    for (uint32_t n = blockIdx.x; n < p.nitems; n += gridDim.x, ++k) {
+        const uint32_t s = k % kStages, use = k / kStages;
+        if (!mbar_wait(&sh.full[s], use & 1u, p.status, kStatusFullTimeout)) break;
+        Stage<DIST> &st = sh.stage[s];
+        const uint32_t i = st.worker, t0 = st.t0, nvalid = st.nvalid, flags = st.flags;
+        float4 xn[kPasses];
+
+        if (!(flags & kItemDistanceOnly)) {
+            const WorkerConst w = p.w[i];
+            if (flags & kItemAverage) {
+                // ---- z (.) hvp in place over the widened range
+                const uint32_t ea0 = st.ea0, ea1 = (st.e1 + 3u) & ~3u, g0 = ea0 >> 7;
+                for (uint32_t q = ctid; q < (ea1 - ea0) >> 2; q += kConsumers) {
+                    const uint32_t j = ea0 + 4u * q;
+                    const uint32_t word = st.zw[(j >> 7) - g0][(j >> 5) & 3u];
+                    float *ptr = &st.hv[j + kHalo - t0];
+                    st_vec(ptr, apply_signs(ld_vec(ptr), (word >> (j & 31u)) & 0xFu));
+                }
+                consumer_sync();
+                // ---- block means in place, one thread per block
+                const uint32_t e0 = st.e0, e1 = st.e1;
+                for (uint32_t ri = st.run0;; ++ri) {
+                    const Run rn = p.runs[ri];
+                    if (rn.start >= e1) break;
+                    if (rn.block > 1u) {
+                        const uint32_t qa = max(e0, rn.start), qb = min(e1, rn.end);
+                        const uint32_t nblk = __umulhi(qb - qa, rn.magic);
+                        float *base = &st.hv[qa + kHalo - t0];
+                        if (rn.block == 9u) block_means_fixed<9>(base, nblk, ctid);
+                        else block_means_any(base, nblk, rn.block, ctid);
                     }
+                    if (rn.end >= e1) break;
                 }
-                if (rn.end >= ti.e1) break;
+                consumer_sync();
             }
-            __syncthreads();
+            float *xr = p.x + (uint64_t)i * p.lds + t0;
+            float *mr = p.m + (uint64_t)i * p.lds + t0;
+            float *vr = p.v + (uint64_t)i * p.lds + t0;
 #pragma unroll
-            for (int r = 0; r < kGroupsPerWarp; ++r)
-                if (nv[r] > 0) dv[r] = ld_vec(&sD[jw + 128u * r - ea0]);
+            for (int pass = 0; pass < kPasses; ++pass) {
+                const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                if (off < nvalid) {
+                    const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
+                    float4 D = ld_vec(&st.hv[off + kHalo]);
+                    if (!(flags & kItemAverage)) {
+                        const uint32_t word = st.zw[off >> 7][(off >> 5) & 3u];
+                        D = apply_signs(D, (word >> (off & 31u)) & 0xFu);
+                    }
+                    const float4 g = ld_vec(&st.g[off]);
+                    float4 x = ld_vec(&st.x[off]), m = ld_vec(&st.m[off]), v = ld_vec(&st.v[off]);
+                    adahessian_update<POWMODE, WD>(x.x, m.x, v.x, g.x, D.x, p, w);
+                    if (nv > 1) adahessian_update<POWMODE, WD>(x.y, m.y, v.y, g.y, D.y, p, w);
+                    if (nv > 2) adahessian_update<POWMODE, WD>(x.z, m.z, v.z, g.z, D.z, p, w);
+                    if (nv > 3) adahessian_update<POWMODE, WD>(x.w, m.w, v.w, g.w, D.w, p, w);
+                    st_vec(xr + off, x);
+                    st_vec(mr + off, m);
+                    st_vec(vr + off, v);
+                    xn[pass] = x;
+                }
+            }
+        } else if constexpr (DIST) {
+#pragma unroll
+            for (int pass = 0; pass < kPasses; ++pass) {
+                const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                if (off < nvalid) xn[pass] = ld_vec(&st.x[off]);
+            }
         }
 
-        // -------- moments and update, then store
+        if constexpr (DIST) {
+            double *red = sh.red[k & 1u];
 #pragma unroll
-        for (int r = 0; r < kGroupsPerWarp; ++r) {
-            if (nv[r] > 0) {
-                const uint32_t j = jw + 128u * r;
-                float4 x = xv[r], m = mv[r], v = vv[r];
-                adahessian_update<POWMODE, WD>(x.x, m.x, v.x, gv[r].x, dv[r].x, p, bc1, bc2);
-                if (nv[r] > 1) adahessian_update<POWMODE, WD>(x.y, m.y, v.y, gv[r].y, dv[r].y, p, bc1, bc2);
-                if (nv[r] > 2) adahessian_update<POWMODE, WD>(x.z, m.z, v.z, gv[r].z, dv[r].z, p, bc1, bc2);
-                if (nv[r] > 3) adahessian_update<POWMODE, WD>(x.w, m.w, v.w, gv[r].w, dv[r].w, p, bc1, bc2);
-                st_vec(xr + j, x);
-                st_vec(mr + j, m);
-                st_vec(vr + j, v);
-                xv[r] = x;
+            for (int pass = 0; pass < kPasses; ++pass) {
+                const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                double d = 0.0;
+                if (off < nvalid) {
+                    const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
+                    d = dist4(xn[pass], ld_vec(&st.c[off]), nv);
+                }
+                d = warp_tree_sum(d);
+                if (lane == 0) red[pass * kConsumerWarps + warp] = d;
+            }
+            consumer_sync();
+            if (ctid == 0) {
+                constexpr int kN = kPasses * kConsumerWarps;
+                double t[kN];
+#pragma unroll
+                for (int q = 0; q < kN; ++q) t[q] = red[q];
+#pragma unroll
+                for (int len = kN; len > 1; len >>= 1)
+#pragma unroll
+                    for (int q = 0; q < len / 2; ++q) t[q] = __dadd_rn(t[2 * q], t[2 * q + 1]);
+                p.partials[(uint64_t)i * p.ntiles_pad + st.tile] = t[0];
             }
         }
-    } else {
-#pragma unroll
-        for (int r = 0; r < kGroupsPerWarp; ++r)
-            if (nv[r] > 0) xv[r] = ld_vec(xr + jw + 128u * r);
-    }
 
-    if (DIST) {
-        double s[kGroupsPerWarp];
-#pragma unroll
-        for (int r = 0; r < kGroupsPerWarp; ++r) {
-            double d = 0.0;
-            if (nv[r] > 0) d = dist4(xv[r], ld_vec(p.c + jw + 128u * r), nv[r]);
-            s[r] = warp_tree_sum(d);
-        }
-#pragma unroll
-        for (int n = kGroupsPerWarp; n > 1; n >>= 1)
-#pragma unroll
-            for (int k = 0; k < n / 2; ++k) s[k] = __dadd_rn(s[2 * k], s[2 * k + 1]);
-        if (lane == 0) sRed[warp] = s[0];
-        __syncthreads();
-        if (tid == 0) {
-            double t[kWarps];
-#pragma unroll
-            for (int k = 0; k < kWarps; ++k) t[k] = sRed[k];
-#pragma unroll
-            for (int n = kWarps; n > 1; n >>= 1)
-#pragma unroll
-                for (int k = 0; k < n / 2; ++k) t[k] = __dadd_rn(t[2 * k], t[2 * k + 1]);
-            p.partials[(uint64_t)i * p.ntiles_pad + tile] = t[0];
-        }
+        // ---- hand the stage back
+        fence_generic_to_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.empty[s]);
     }
 }
 
@@ -371,26 +528,46 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-template <int POWMODE, bool WD>
-static cudaError_t launch_step_dist(const StepParams &p, dim3 grid, bool want_dist, cudaStream_t s)
+template <int POWMODE, bool WD, bool DIST>
+static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream_t s)
 {
-    if (want_dist) local_step_kernel<POWMODE, WD, true><<<grid, kThreads, 0, s>>>(p);
-    else           local_step_kernel<POWMODE, WD, false><<<grid, kThreads, 0, s>>>(p);
+    auto kernel = local_step_kernel<POWMODE, WD, DIST>;
+    const size_t smem = sizeof(Shared<DIST>);
+    static bool configured = false;      // per instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (p.nitems == 0) return cudaSuccess;
+    const uint32_t resident = (uint32_t)sm_count * (uint32_t)kCtasPerSm;
+    const uint32_t grid = p.nitems < resident ? p.nitems : resident;
+    kernel<<<grid, kThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_local_step(const StepParams &p, int K, bool want_dist, cudaStream_t s)
+template <int POWMODE, bool WD>
+static cudaError_t launch_step_dist(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
 {
-    const dim3 grid(p.ntiles, (unsigned)K);
+    return want_dist ? launch_step_one<POWMODE, WD, true>(p, sm_count, s)
+                     : launch_step_one<POWMODE, WD, false>(p, sm_count, s);
+}
+
+cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
+{
     const int mode = p.hpow == 1.0f ? 0 : (p.hpow == 0.5f ? 1 : 2);
     const bool wd = p.wd != 0.0f;
     switch (mode * 2 + (wd ? 1 : 0)) {
-    case 0: return launch_step_dist<0, false>(p, grid, want_dist, s);
-    case 1: return launch_step_dist<0, true>(p, grid, want_dist, s);
-    case 2: return launch_step_dist<1, false>(p, grid, want_dist, s);
-    case 3: return launch_step_dist<1, true>(p, grid, want_dist, s);
-    case 4: return launch_step_dist<2, false>(p, grid, want_dist, s);
-    default: return launch_step_dist<2, true>(p, grid, want_dist, s);
+    case 0: return launch_step_dist<0, false>(p, want_dist, sm_count, s);
+    case 1: return launch_step_dist<0, true>(p, want_dist, sm_count, s);
+    case 2: return launch_step_dist<1, false>(p, want_dist, sm_count, s);
+    case 3: return launch_step_dist<1, true>(p, want_dist, sm_count, s);
+    case 4: return launch_step_dist<2, false>(p, want_dist, sm_count, s);
+    default: return launch_step_dist<2, true>(p, want_dist, sm_count, s);
     }
 }
 

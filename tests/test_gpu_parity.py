@@ -28,7 +28,7 @@ def torch():
     return torch
 
 
-ODD_SEGS = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 256)]
+ODD_SEGS = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 128)]
 ODD_P = 13_111
 
 
@@ -66,7 +66,7 @@ def test_sample_z_bit_exact(B, torch, K, P):
     ([(0, 5000, 1)], 5000),                      # one unstructured tensor
     ([], 2048 * 3),                              # no table at all, exact tiles
     ([(0, 9 * 700, 9)], 6300),                   # blocks straddle tile edges
-    (ODD_SEGS, ODD_P),                           # odd offsets, gaps, block 49/5/256
+    (ODD_SEGS, ODD_P),                           # odd offsets, gaps, block 49/5/128
     ([(0, 1, 1)], 1), ([(0, 3, 3)], 3), ([(1, 4, 2)], 6),
 ])
 @pytest.mark.parametrize("hp,wd", [(1.0, 0.0), (0.5, 0.01), (0.75, 0.0)])

@@ -55,11 +55,11 @@ def test_status_strings_and_argument_checks(B):
     ([(9, 9, 9), (0, 9, 9)], "SEGMENTS"),  # unsorted
     ([(0, 200, 1)], "SEGMENTS"),           # beyond P
     ([(0, 0, 0)], "SEGMENTS"),             # block 0
-    ([(0, 514, 257)], "SEGMENTS"),         # block above the maximum
+    ([(0, 258, 129)], "SEGMENTS"),         # block above the maximum
 ])
 def test_bad_segment_tables_are_rejected(B, segs, code):
     with pytest.raises(B.AdaHessError) as e:
-        B.Handle(2, 100 if segs[0][1] != 514 else 1000, segs, host_only=True)
+        B.Handle(2, 100 if segs[0][1] != 258 else 1000, segs, host_only=True)
     assert e.value.status == getattr(B, "AH_ERR_" + code)
 
 
@@ -107,7 +107,7 @@ def test_weights_match_oracle_bit_for_bit_given_same_distances(B):
 @pytest.mark.parametrize("name", ["resnet18", "resnet50", "vgg16", "odd"])
 def test_tile_descriptors_cover_whole_blocks(B, name):
     if name == "odd":
-        segs = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 256)]
+        segs = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 128)]
         P = 13_111
     else:
         layout = W.LAYOUTS[name](8)
