@@ -52,7 +52,8 @@ HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weigh
 # DRAM bytes per parameter update of the fused local-step kernel, from one ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch / (K * P)), and the hash
 # of the kernel sources it was taken on.  Reported only while the sources are unchanged.
-NCU_TRAFFIC = {"sources_sha256": None, "dram_bytes_per_update": None}
+NCU_TRAFFIC = {"sources_sha256": "1cca58c8068d2b49fe52e249e8e5b7055ba94e780a9c2b2bba29f2f657b99434",
+               "dram_bytes_per_update": 1.446244e9 / 46_758_048}
 
 
 def kernel_sources_hash() -> str:
@@ -131,10 +132,12 @@ class ClockSampler:
 def run_period(h, pool, t0, wl, events=None, stage=None):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
-    memory (the end-to-end leg).  Returns bytes moved by the local-step launches."""
+    memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
+    exchanged)."""
     import torch
     _, K, tau, p_fail, max_stale, frozen = wl
     alpha = alpha_for(K)
+    worker_steps = exchanged = 0
     for r in range(tau):
         t = t0 + r + 1
         mask = h.dw_mask_next(MASK_SEED, t, p_fail, max_stale)
@@ -151,14 +154,16 @@ def run_period(h, pool, t0, wl, events=None, stage=None):
             e0.record()
         h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
                         **HYPER)
+        n_act = int(mask.sum()) if frozen else K
+        worker_steps += n_act
         if events is not None:
             e1.record()
-            n_act = int(mask.sum()) if frozen else K
             events.append((e0, e1, ex, n_act))
         if ex:
             w = h.dw_weights_next(alpha)
             h.easgd_exchange(mask, w, alpha)
-    return t0 + tau
+            exchanged += int(mask.sum())
+    return t0 + tau, worker_steps, exchanged
 
 
 def gpu_arm(args):
@@ -199,7 +204,7 @@ def gpu_arm(args):
 
     t = 0
     for _ in range(args.warmup):
-        t = run_period(h, pool, t, wl)
+        t, _, _ = run_period(h, pool, t, wl)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -208,8 +213,11 @@ def gpu_arm(args):
     events = []
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
+    worker_steps = exchanged = 0
     for _ in range(args.steps):
-        t = run_period(h, pool, t, wl, events)
+        t, ws, exd = run_period(h, pool, t, wl, events)
+        worker_steps += ws
+        exchanged += exd
     stop.record()
     barrier()
     ms = start.elapsed_time(stop)
@@ -219,16 +227,23 @@ def gpu_arm(args):
         tmax = torch.tensor([ms], device=dev)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         ms = float(tmax.item())
-    updates = K * P * tau * args.steps * world
+    # parameter updates actually performed: a frozen straggler takes no step
+    updates = worker_steps * P * world
     value = updates / (ms * 1e-3) / 1e9
 
     # per-launch duration of the fused local-step kernel (plain rounds; the rounds that
     # also measure distances are listed beside it)
     plain = [(a.elapsed_time(b), n) for a, b, ex, n in events if not ex]
     withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex]
-    dom, extra_bytes, dom_name = (plain, 0, "local_step") if plain else (withd, 4 * P, "local_step+dist")
+    # algorithmic bytes of a launch: 32 per update; a distance round also reads the
+    # master row once and the x of every worker that sat the step out
+    if plain:
+        dom, dom_name = plain, "local_step"
+        dom_bytes = sum(32 * P * n for _, n in dom) / len(dom)
+    else:
+        dom, dom_name = withd, "local_step+dist"
+        dom_bytes = sum(32 * P * n + 4 * P * (K - n) + 4 * P for _, n in dom) / len(dom)
     dom_ms = sum(d for d, _ in dom) / len(dom)
-    dom_bytes = sum(32 * P * n + extra_bytes for _, n in dom) / len(dom)
     peak, peak_kind = measured_hbm_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
@@ -239,9 +254,9 @@ def gpu_arm(args):
                 "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": traffic,
                 "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
                 "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
-    # whole-period bytes: 32 per update + (8 K_act P + 12 P) per exchange
-    period_bytes = 32 * K * P * tau + 8 * K * P + 12 * P
-    whole = {"algorithmic_GBps": round(period_bytes * args.steps / (ms * 1e-3) / 1e9, 1)}
+    # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
+    run_bytes = 32 * P * worker_steps + 8 * P * exchanged + 12 * P * args.steps
+    whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
 
     # end-to-end leg: same periods, inputs copied from pinned host memory every round,
@@ -252,11 +267,13 @@ def gpu_arm(args):
         host_pool = [(g.cpu().pin_memory(), hv.cpu().pin_memory()) for g, hv in pool[:n_host]]
         sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
-        t = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
         barrier()
         start.record()
+        e2e_ws = 0
         for _ in range(e2e_steps):
-            t = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+            e2e_ws += ws
         stop.record()
         barrier()
         ems = start.elapsed_time(stop)
@@ -264,7 +281,7 @@ def gpu_arm(args):
             tmax = torch.tensor([ems], device=dev)
             dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
             ems = float(tmax.item())
-        e2e = {"value": round(K * P * tau * e2e_steps * world / (ems * 1e-3) / 1e9, 3),
+        e2e = {"value": round(e2e_ws * P * world / (ems * 1e-3) / 1e9, 3),
                "unit": "G param-updates/s", "steps": e2e_steps,
                "h2d_bytes_per_step": pair_bytes * tau, "d2h_bytes_per_step": 8 * K}
 
@@ -278,6 +295,7 @@ def gpu_arm(args):
                                f"p_fail={p_fail}, max_stale={max_stale}, frozen_stragglers={frozen}",
                    "step": f"one communication period = {tau} rounds + 1 exchange",
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
+                   "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
                          % ((32 * K * P) / 1e9) if 32 * K * P > 4 * 126e6 else
                          "working set comparable to L2: partly L2-resident, reported as is",
@@ -314,7 +332,8 @@ def oracle_sample(args, max_params):
 
 
 def oracle_periods(args, layout, periods, warm):
-    """Runs warm + periods communication periods of the oracle; returns (seconds, K, P, tau, threads)."""
+    """Runs warm + periods communication periods of the oracle; returns (seconds, K, P, tau,
+    threads, worker-steps taken in the timed periods)."""
     import numpy as np
     from paper_2409_09242_b200 import workloads as W
     kind, K, tau, p_fail, max_stale, frozen = WORKLOADS[args.workload]
@@ -325,29 +344,31 @@ def oracle_periods(args, layout, periods, warm):
     pool = W.gaussian_pool_np(layout, K, 2, DATA_SEED + 1)
     st = oracle.OracleState(W.theta0_np(layout, DATA_SEED), K, segs, variant="omp")
     alpha = alpha_for(K)
-    t, t_start = 0, None
+    t, t_start, worker_steps = 0, None, 0
     for period in range(warm + periods):
         if period == warm:
             t_start = time.perf_counter()
         for r in range(tau):
             t += 1
             mask = st.mask_next(MASK_SEED, t, p_fail, max_stale)
+            if period >= warm:
+                worker_steps += int(mask.sum()) if frozen else K
             ex = r == tau - 1
             g, hv = pool[t % 2]
             st.local_step(g, hv, Z_SEED, t, active=mask if frozen else None, want_dist=ex, **HYPER)
             if ex:
                 h2, h1 = st.weights_next(alpha)
                 st.exchange(mask, h2, h1)
-    return time.perf_counter() - t_start, K, P, tau, min(threads, st.o.num_threads())
+    return time.perf_counter() - t_start, K, P, tau, min(threads, st.o.num_threads()), worker_steps
 
 
 def cpu_baseline(args, budget_s):
     """The CPU oracle, as it stands, timed on this host on a bounded sample."""
     layout, what = oracle_sample(args, max_params=4_000_000)
-    sec, K, P, tau, threads = oracle_periods(args, layout, periods=1, warm=0)
-    periods = max(1, min(20, int(budget_s / max(sec, 1e-3))))
-    sec, K, P, tau, threads = oracle_periods(args, layout, periods=periods, warm=1)
-    return {"value": round(K * P * tau * periods / sec / 1e9, 5), "unit": "G param-updates/s",
+    sec, K, P, tau, threads, _ = oracle_periods(args, layout, periods=1, warm=1)
+    periods = max(1, min(200, int(budget_s / max(sec, 1e-3))))
+    sec, K, P, tau, threads, ws = oracle_periods(args, layout, periods=periods, warm=1)
+    return {"value": round(ws * P / sec / 1e9, 5), "unit": "G param-updates/s",
             "cores": threads, "kind": "oracle",
             "sample": f"{what}; {periods} periods of {tau} rounds, {sec:.1f} s; OpenMP build, "
                       f"local steps parallel over workers ({threads} threads)"}
@@ -358,8 +379,8 @@ def reference_arm(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     layout, what = oracle_sample(args, max_params=1_000_000)
-    sec, K, P, tau, threads = oracle_periods(args, layout, periods=args.steps, warm=args.warmup)
-    value = round(K * P * tau * args.steps / sec / 1e9, 5)
+    sec, K, P, tau, threads, ws = oracle_periods(args, layout, periods=args.steps, warm=args.warmup)
+    value = round(ws * P / sec / 1e9, 5)
     kind = WORKLOADS[args.workload][0]
     print(json.dumps({
         "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
