@@ -48,11 +48,13 @@ extern "C" {
 #define AH_ERR_STATE         (-6)  /* call out of order (e.g. weights asked for before a
                                       step with want_dist = 1 produced the distances)      */
 #define AH_ERR_INTERNAL      (-7)  /* the device status word was set by a kernel            */
+#define AH_ERR_TOO_LARGE     (-8)  /* problem exceeds a fixed capacity (ah_distances_static) */
 
 #define AH_MAX_WORKERS  256        /* K <= 256                                              */
 #define AH_MAX_BLOCK    128        /* spatial block kh*kw <= 128 (covers 11 x 11 kernels)   */
 #define AH_MAX_HIST     32         /* history depth p of the raw score <= 32                */
 #define AH_ROUND_AUTO   0xFFFFFFFFu
+#define AH_STATIC_SCRATCH_ENTRIES (1 << 17)  /* doubles per row of the built-in scratch     */
 #define AH_DEVICE_NONE  (-2)       /* ah_alloc.device: bookkeeping-only handle, no GPU      */
 
 /* ---- types ---------------------------------------------------------------- */
@@ -221,6 +223,35 @@ int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int ma
  * weights: host pointer, 2K floats as written by dw_weights_next, or NULL
  * (h1_i = h2_i = alpha for all i).  alpha is ignored when weights != NULL. */
 int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha);
+
+/* ---- without a handle, without allocating ------------------------------------ */
+
+/* (No counterpart in the paper: a deployment convenience.)
+ * norm2[i] = ||x_i - c||^2 for i = 0..K-1, the same quantity, summed in the same
+ * pairwise order and therefore bit-identical to what a want_dist step leaves in a
+ * handle, for callers that hold raw pointers and must not allocate: a hook running
+ * inside a job whose framework has already claimed the whole GPU, a
+ * latency-critical loop that cannot afford the device-wide synchronisation of an
+ * allocation, or a component with no ah_ctx of its own (ah_init allocates).  The
+ * call makes no cudaMalloc/cudaFree and uses no workspace: its per-tile partial sums
+ * go to a fixed 2 MiB array that is part of the library image on every GPU that
+ * loads it.
+ *   x      device pointer, [K][ldx] binary32, ldx >= P, ldx % 4 == 0, 16-byte aligned
+ *   c      device pointer, [P] binary32, 16-byte aligned, readable up to P rounded up to 4
+ *   norm2  device pointer, K doubles, written when the stream reaches the kernels
+ *   cuda_stream  cudaStream_t or NULL; the call returns without waiting
+ * The device that owns the pointers must be the current device.
+ * Capacity: K * (ceil(P / 1024) rounded up to a power of two) <=
+ * AH_STATIC_SCRATCH_ENTRIES (for example K = 4 with P up to 33.5 M, or K = 16 with P
+ * up to 8.3 M); beyond it the call returns AH_ERR_TOO_LARGE and does nothing.
+ * The first call on each device looks up the array's device address (a runtime
+ * query, no allocation); make that first call outside any stream capture.
+ * All calls share the one array and it keeps the previous call's contents; nothing
+ * in it needs clearing, but two calls whose kernels may overlap on the GPU (other
+ * streams, other threads) race on it: serialise them.
+ * Errors: INVALID_ARG, ALIGN, TOO_LARGE, CUDA. */
+int ah_distances_static(const float *x, uint64_t ldx, const float *c, int K, uint64_t P,
+                        double *norm2, void *cuda_stream);
 
 /* ---- diagnostics ------------------------------------------------------------- */
 const char *ah_status_string(int status);

@@ -24,7 +24,8 @@ _lib = C.CDLL(_build.LIB_PATH)
 
 AH_OK = 0
 AH_ERR_INVALID_ARG, AH_ERR_ALIGN, AH_ERR_SEGMENTS, AH_ERR_ALLOC = -1, -2, -3, -4
-AH_ERR_CUDA, AH_ERR_STATE, AH_ERR_INTERNAL = -5, -6, -7
+AH_ERR_CUDA, AH_ERR_STATE, AH_ERR_INTERNAL, AH_ERR_TOO_LARGE = -5, -6, -7, -8
+AH_STATIC_SCRATCH_ENTRIES = 1 << 17
 AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST = 256, 128, 32
 AH_ROUND_AUTO = 0xFFFFFFFF
 AH_DEVICE_NONE = -2
@@ -33,7 +34,7 @@ AH_DEVICE_NONE = -2
 
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_local_step", "dw_config",
-           "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange", "ah_status_string",
+           "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -69,6 +70,7 @@ _lib.dw_weights_from_norm2.argtypes = [_vp, C.POINTER(C.c_double), C.c_float, C.
 _lib.dw_mask_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_double, C.c_int,
                               C.POINTER(C.c_uint8)]
 _lib.easgd_exchange.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float]
+_lib.ah_distances_static.argtypes = [_vp, C.c_uint64, _vp, C.c_int, C.c_uint64, _vp, _vp]
 _lib.ah_status_string.argtypes = [C.c_int]
 _lib.ah_status_string.restype = C.c_char_p
 _lib.ah_last_cuda_error.argtypes = [_vp]
@@ -106,6 +108,26 @@ def _segments(segments):
     for k, s in enumerate(segments):
         arr[k] = ah_segment(int(s[0]), int(s[1]), int(s[2]), 0)
     return arr
+
+
+def ah_distances_static(x, c, norm2_out, stream=None):
+    """||x_i - c||^2 for raw tensors, no handle, no allocation inside the library.
+
+    x: float32 CUDA tensor [K, ld] (rows contiguous), c: float32 CUDA tensor with at
+    least P = x.shape[1] entries (padded to a multiple of 4), norm2_out: float64 CUDA
+    tensor [K], written asynchronously on `stream` (default: torch's current stream).
+    The caller provides every buffer, the output included."""
+    import torch
+    K, P = x.shape
+    if norm2_out.dtype != torch.float64 or not norm2_out.is_cuda or norm2_out.numel() < K:
+        raise TypeError("norm2_out: float64 CUDA tensor of K entries")
+    if stream is None:
+        stream = torch.cuda.current_stream(x.device).cuda_stream
+    rc = _lib.ah_distances_static(_dev_ptr(x, "x"), x.stride(0), _dev_ptr(c, "c"), int(K), int(P),
+                                  norm2_out.data_ptr(), stream)
+    if rc != AH_OK:
+        raise AdaHessError(rc, "ah_distances_static")
+    return norm2_out
 
 
 def raw():

@@ -559,6 +559,7 @@ const char *ah_status_string(int status)
     case AH_ERR_CUDA: return "CUDA runtime error";
     case AH_ERR_STATE: return "call out of order";
     case AH_ERR_INTERNAL: return "internal device error";
+    case AH_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity";
     default: return "unknown status";
     }
 }
