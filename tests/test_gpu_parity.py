@@ -336,3 +336,80 @@ def test_error_paths_and_own_allocation(B, torch):
     out = C.c_void_p(None)
     assert lib.ah_init(C.byref(out), 4, 10_000, None, 0, C.byref(opt)) == B.AH_ERR_ALLOC
     assert out.value is None
+
+
+# ------------------------------------------- full-size configurations, short runs
+def _full_size_run(B, kind, K, tau, rounds, p_fail, max_stale=1, frozen=False, n_pool=1):
+    layout = W.LAYOUTS[kind]()
+    cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=rounds,
+                    tau=tau, p_fail=p_fail, max_stale=max_stale, frozen=frozen)
+    _check_run(B, cfg, _layout_inputs(layout, K, n_pool=n_pool))
+
+
+def test_full_size_resnet18_layout(B, torch):
+    # config 2 at its full size (P = 11,689,512, K = 8): two communication periods
+    _full_size_run(B, "resnet18", 8, 4, 8, 0.1, n_pool=2)
+
+
+def test_full_size_resnet50_layout_stragglers(B, torch):
+    # config 3 at its full size (P = 25,557,032, K = 16), frozen stragglers
+    _full_size_run(B, "resnet50", 16, 4, 4, 0.2, max_stale=8, frozen=True)
+
+
+def test_full_size_vgg16_layout(B, torch):
+    # config 4 at its full size (P = 138,357,544, K = 4, tau = 8): one period
+    _full_size_run(B, "vgg16", 4, 8, 8, 0.25)
+
+
+def test_full_size_k64_prefix_sample_and_distance_property(B, torch):
+    """Config 5's largest case (ResNet-50-shaped layout, K = 64, 19.6 GB of state) in the
+    launch shape the bench times.  The oracle recomputes a sample it can afford: every
+    worker's leading tensors (columns are independent given the masks and a fixed alpha,
+    and z is indexed by absolute position), compared element by element; the full-size
+    distances are checked against a double-precision sum formed on the device."""
+    layout = W.resnet50_layout()
+    segs, P, K, tau, R = W.segments(layout), W.total_params(layout), 64, 4, 8
+    ld = W.padded_ld(P)
+    n_keep = next(k for k, tns in enumerate(layout) if tns.offset + tns.numel > 1_500_000)
+    prefix = layout[:n_keep]
+    Pp = W.total_params(prefix)
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    g = torch.empty((K, ld), device="cuda").normal_(generator=gen).mul_(0.05)
+    hv = torch.empty((K, ld), device="cuda").normal_(generator=gen).mul_(0.05)
+    theta0 = torch.empty(P, device="cuda").normal_(generator=gen).mul_(0.05)
+    h = B.Handle(K, P, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    gp = np.ascontiguousarray(g[:, :Pp].cpu().numpy())
+    hp = np.ascontiguousarray(hv[:, :Pp].cpu().numpy())
+    ref = OracleState(theta0[:Pp].cpu().numpy(), K, W.segments(prefix), variant="omp")
+    alpha = 0.8 / K
+    from parity_driver import MASK_SEED
+    for t in range(1, R + 1):
+        mask = h.dw_mask_next(MASK_SEED, t, 0.1)
+        assert np.array_equal(mask, ref.mask_next(MASK_SEED, t, 0.1))
+        ex = t % tau == 0
+        h.ah_local_step(g, hv, Z_SEED, lr=0.01, round_=t, want_dist=ex)
+        ref.local_step(gp, hp, Z_SEED, t, lr=0.01)
+        if ex:
+            # distances at full size: same value as a double-precision sum on the device
+            xs = torch.empty((K, P), device="cuda")
+            cs = torch.empty(P, device="cuda")
+            h.ah_state_get(B.AH_X, out=xs)
+            h.ah_state_get(B.AH_CENTER, out=cs)
+            n2 = h.ah_state_get(B.AH_NORM2)
+            for i in (0, 17, 63):
+                want = float(((xs[i] - cs).double() ** 2).sum().item())
+                assert abs(n2[i] - want) <= 1e-11 * want, (t, i)
+            del xs, cs
+            h.easgd_exchange(mask, None, alpha)
+            ref.exchange(mask, alpha=alpha)
+    row = torch.empty(P, device="cuda")
+    for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v)):
+        for i in range(K):
+            h.ah_state_get(which, worker=i, out=row)
+            got = row[:Pp].cpu().numpy()
+            assert np.array_equal(got.view(np.uint32), want[i].view(np.uint32)), (which, i)
+    h.ah_state_get(B.AH_CENTER, out=row)
+    assert np.array_equal(row[:Pp].cpu().numpy().view(np.uint32), ref.center.view(np.uint32))
+    h.close()
