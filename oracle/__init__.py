@@ -108,6 +108,11 @@ class Oracle:
         L.orc_mask_next.restype = None
         L.orc_exchange.argtypes = [pf, pf, C.c_int, C.c_uint64, pu8, pf, pf]
         L.orc_exchange.restype = None
+        pu16 = C.POINTER(C.c_uint16)
+        L.orc_exchange_async.argtypes = [pf, pf, C.c_int, C.c_uint64, pu8, pf, pf, pu16, C.c_int]
+        L.orc_exchange_async.restype = None
+        L.orc_order_next.argtypes = [C.c_int, C.c_uint64, C.c_uint32, pu16]
+        L.orc_order_next.restype = None
         L.orc_is_double.restype = C.c_int
         L.orc_num_threads.restype = C.c_int
 
@@ -152,6 +157,19 @@ class Oracle:
     def exchange(self, x, xc, mask, h2, h1):
         K, P = x.shape
         self.lib.orc_exchange(_f32(x), _f32(xc), K, P, _u8(mask), _f32(h2), _f32(h1))
+
+    def exchange_async(self, x, xc, mask, h2, h1, order=None):
+        K, P = x.shape
+        n, po = 0, None
+        if order is not None:
+            order = np.ascontiguousarray(order, np.uint16)
+            n, po = order.size, order.ctypes.data_as(C.POINTER(C.c_uint16))
+        self.lib.orc_exchange_async(_f32(x), _f32(xc), K, P, _u8(mask), _f32(h2), _f32(h1), po, n)
+
+    def order_next(self, K, seed, t):
+        order = np.empty(K, np.uint16)
+        self.lib.orc_order_next(K, int(seed), int(t), order.ctypes.data_as(C.POINTER(C.c_uint16)))
+        return order
 
     def num_threads(self):
         return int(self.lib.orc_num_threads())
@@ -244,3 +262,16 @@ class OracleState:
             mask = np.ascontiguousarray(mask, np.uint8)
         self.o.exchange(self.x, self.center, mask, np.ascontiguousarray(h2, np.float32),
                         np.ascontiguousarray(h1, np.float32))
+
+    # asynchronous form of S6: workers arrive one at a time in `order`
+    def exchange_async(self, mask=None, h2=None, h1=None, alpha=0.0, order=None):
+        if h2 is None:
+            h2 = np.full(self.K, alpha, np.float32)
+            h1 = np.full(self.K, alpha, np.float32)
+        if mask is not None:
+            mask = np.ascontiguousarray(mask, np.uint8)
+        self.o.exchange_async(self.x, self.center, mask, np.ascontiguousarray(h2, np.float32),
+                              np.ascontiguousarray(h1, np.float32), order)
+
+    def order_next(self, seed, t):
+        return self.o.order_next(self.K, seed, t)

@@ -381,6 +381,55 @@ void orc_exchange(float *x, float *xc, int K, uint64_t P, const uint8_t *mask,
     }
 }
 
+/* ------------------------------------------------------------------------- */
+/* Asynchronous form of the exchange.  Sec. II assumes asynchronous training and
+ * Eqs. 12-13 are written for one worker talking to the master: the workers reach
+ * the master one at a time, and each one sees the master as the workers before it
+ * left it.  order[0..n_order) lists the workers in the order in which they arrive
+ * (NULL = 0, 1, ..., K-1); a worker whose mask byte is 0 does not arrive.  For
+ * every column j:
+ *   c = xc_j
+ *   for q ascending, i = order[q], mask_i: d = x_ij - c; x_ij -= h1_i d; c += h2_i d
+ *   xc_j = c                                                                      */
+/* ------------------------------------------------------------------------- */
+void orc_exchange_async(float *x, float *xc, int K, uint64_t P, const uint8_t *mask,
+                        const float *h2, const float *h1, const uint16_t *order, int n_order)
+{
+    const int n = order ? n_order : K;
+#pragma omp parallel for schedule(static)
+    for (uint64_t j = 0; j < P; ++j) {
+        real c = (real)xc[j];
+        for (int q = 0; q < n; ++q) {
+            const int i = order ? (int)order[q] : q;
+            if (mask && !mask[i]) continue;
+            float *xi = x + (uint64_t)i * P;
+            const real d = (real)xi[j] - c;
+            xi[j] = (float)((real)xi[j] - ((real)h1[i] * d));
+            c = (real)(float)(c + ((real)h2[i] * d));
+        }
+        xc[j] = (float)c;
+    }
+}
+
+/* Seeded arrival order of round t: a uniformly random permutation of 0..K-1 by the
+ * Fisher-Yates shuffle (Durstenfeld's form), driven by the counter-based generator:
+ * start from the identity; for q = K-1 down to 1 draw
+ * r = Philox(seed; (q, 0, t, 3))[0] and swap entries q and r mod (q+1).           */
+enum { ORC_DOMAIN_ORDER = 3 };
+
+void orc_order_next(int K, uint64_t seed, uint32_t t, uint16_t *order)
+{
+    uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    for (int i = 0; i < K; ++i) order[i] = (uint16_t)i;
+    for (int q = K - 1; q >= 1; --q) {
+        uint32_t ctr[4] = { (uint32_t)q, 0u, t, ORC_DOMAIN_ORDER };
+        uint32_t r[4];
+        orc_philox4x32_10(ctr, key, r);
+        const uint32_t pick = r[0] % (uint32_t)(q + 1);
+        const uint16_t tmp = order[q]; order[q] = order[pick]; order[pick] = tmp;
+    }
+}
+
 int orc_is_double(void)
 {
 #ifdef ORC_DOUBLE
