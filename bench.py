@@ -29,7 +29,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-Z_SEED, MASK_SEED, DATA_SEED = 0x5EED0001, 0x5EED0002, 0
+Z_SEED, MASK_SEED, ORDER_SEED, DATA_SEED = 0x5EED0001, 0x5EED0002, 0x5EED0003, 0
 
 # name -> (layout, K, tau, p_fail, max_stale, frozen stragglers)
 WORKLOADS = {
@@ -129,7 +129,7 @@ class ClockSampler:
                 "samples": len(clocks), "reasons": sorted(reasons)}
 
 
-def run_period(h, pool, t0, wl, events=None, stage=None):
+def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
     memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
@@ -161,7 +161,16 @@ def run_period(h, pool, t0, wl, events=None, stage=None):
             events.append((e0, e1, ex, n_act))
         if ex:
             w = h.dw_weights_next(alpha)
-            h.easgd_exchange(mask, w, alpha)
+            if ex_events is not None:
+                x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                x0.record()
+            if asynchronous:
+                h.easgd_exchange_async(mask, w, alpha, h.dw_order_next(ORDER_SEED, t))
+            else:
+                h.easgd_exchange(mask, w, alpha)
+            if ex_events is not None:
+                x1.record()
+                ex_events.append((x0, x1, int(mask.sum())))
             exchanged += int(mask.sum())
     return t0 + tau, worker_steps, exchanged
 
@@ -203,19 +212,20 @@ def gpu_arm(args):
             torch.cuda.synchronize()
 
     t = 0
+    asyn = args.exchange == "async"
     for _ in range(args.warmup):
-        t, _, _ = run_period(h, pool, t, wl)
+        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     launches0 = h.ah_launch_count()
-    events = []
+    events, ex_events = [], []
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
     worker_steps = exchanged = 0
     for _ in range(args.steps):
-        t, ws, exd = run_period(h, pool, t, wl, events)
+        t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events)
         worker_steps += ws
         exchanged += exd
     stop.record()
@@ -258,6 +268,15 @@ def gpu_arm(args):
     run_bytes = 32 * P * worker_steps + 8 * P * exchanged + 12 * P * args.steps
     whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
+    # the exchange kernel alone: 8 bytes per (arriving worker, parameter) + 8 per parameter
+    exl = [(a.elapsed_time(b), n) for a, b, n in ex_events if n > 0]
+    exchange = None
+    if exl:
+        ex_ms = sum(d for d, _ in exl) / len(exl)
+        ex_bytes = sum(8 * P * n + 8 * P for _, n in exl) / len(exl)
+        exchange = {"kernel": "exchange_async" if asyn else "exchange", "ms_per_launch": round(ex_ms, 4),
+                    "algorithmic_GBps": round(ex_bytes / (ex_ms * 1e-3) / 1e9, 1),
+                    "note": "x was just written by the local step, part of it is still in L2"}
 
     # end-to-end leg: same periods, inputs copied from pinned host memory every round,
     # the distances/weights read back every period
@@ -267,12 +286,12 @@ def gpu_arm(args):
         host_pool = [(g.cpu().pin_memory(), hv.cpu().pin_memory()) for g, hv in pool[:n_host]]
         sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
-        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn)
         barrier()
         start.record()
         e2e_ws = 0
         for _ in range(e2e_steps):
-            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh))
+            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn)
             e2e_ws += ws
         stop.record()
         barrier()
@@ -294,13 +313,14 @@ def gpu_arm(args):
         "config": {"workload": f"{args.workload}: {kind} layout, P={P}, K={K}, tau={tau}, "
                                f"p_fail={p_fail}, max_stale={max_stale}, frozen_stragglers={frozen}",
                    "step": f"one communication period = {tau} rounds + 1 exchange",
+                   "exchange": "asynchronous, seeded arrival order" if asyn else "simultaneous",
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
                    "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
                          % ((32 * K * P) / 1e9) if 32 * K * P > 4 * 126e6 else
                          "working set comparable to L2: partly L2-resident, reported as is",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "roofline": roofline, "whole_step": whole, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "whole_step": whole, "exchange_kernel": exchange, "e2e": e2e, "gpu_launches": int(launches),
         "clocks": clocks,
     }
     h.close()
@@ -358,7 +378,10 @@ def oracle_periods(args, layout, periods, warm):
             st.local_step(g, hv, Z_SEED, t, active=mask if frozen else None, want_dist=ex, **HYPER)
             if ex:
                 h2, h1 = st.weights_next(alpha)
-                st.exchange(mask, h2, h1)
+                if args.exchange == "async":
+                    st.exchange_async(mask, h2, h1, order=st.order_next(ORDER_SEED, t))
+                else:
+                    st.exchange(mask, h2, h1)
     return time.perf_counter() - t_start, K, P, tau, min(threads, st.o.num_threads()), worker_steps
 
 
@@ -401,11 +424,13 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--pool", type=int, default=4, help="grad/hvp pairs kept in HBM")
+    ap.add_argument("--exchange", default="simultaneous", choices=["simultaneous", "async"],
+                    help="all workers against the same master value, or one at a time")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

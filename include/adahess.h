@@ -224,6 +224,30 @@ int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int ma
  * (h1_i = h2_i = alpha for all i).  alpha is ignored when weights != NULL. */
 int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha);
 
+/* ---- asynchronous exchange ---------------------------------------------------- */
+
+/* Seeded arrival order for an asynchronous exchange round (Sec. II: training is
+ * asynchronous, so the workers do not reach the master together): a uniformly random
+ * permutation of 0..K-1, order[q] = the worker that arrives q-th.  Fisher-Yates shuffle
+ * of the identity: for q = K-1 down to 1, entries q and r mod (q+1) trade places,
+ * r = first word of Philox4x32-10 with key (seed low, seed high) and counter
+ * (q, 0, round, 3).  order: host pointer, K entries.  Host-only; touches no GPU. */
+int dw_order_next(ah_ctx *h, uint64_t seed, uint32_t round, uint16_t *order);
+
+/* Weighted elastic exchange with the workers reaching the master one at a time
+ * (Eqs. 12-13 applied per worker, as printed): each arrival sees the master as the
+ * arrivals before it left it.  For every column j:
+ *     c = center_j
+ *     for q = 0..K-1, i = order[q], worker_mask[i] != 0:
+ *         d = x_ij - c;   x_ij -= h1_i * d;   c += h2_i * d
+ *     center_j = c
+ * order: host pointer, K entries naming every worker exactly once (else INVALID_ARG),
+ * or NULL for 0, 1, ..., K-1.  worker_mask, weights, alpha as in easgd_exchange.
+ * Unlike the simultaneous form this stays a contraction for any K (no bound on the
+ * sum of the h2_i).  Same memory traffic as easgd_exchange. */
+int easgd_exchange_async(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
+                         const uint16_t *order);
+
 /* ---- without a handle, without allocating ------------------------------------ */
 
 /* (No counterpart in the paper: a deployment convenience.)

@@ -34,7 +34,8 @@ AH_DEVICE_NONE = -2
 
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_local_step", "dw_config",
-           "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange", "ah_distances_static", "ah_status_string",
+           "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
+           "dw_order_next", "easgd_exchange_async", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -70,6 +71,9 @@ _lib.dw_weights_from_norm2.argtypes = [_vp, C.POINTER(C.c_double), C.c_float, C.
 _lib.dw_mask_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_double, C.c_int,
                               C.POINTER(C.c_uint8)]
 _lib.easgd_exchange.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float]
+_lib.dw_order_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.POINTER(C.c_uint16)]
+_lib.easgd_exchange_async.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
+                                      C.POINTER(C.c_uint16)]
 _lib.ah_distances_static.argtypes = [_vp, C.c_uint64, _vp, C.c_int, C.c_uint64, _vp, _vp]
 _lib.ah_status_string.argtypes = [C.c_int]
 _lib.ah_status_string.restype = C.c_char_p
@@ -311,6 +315,29 @@ class Handle:
                 raise ValueError("weights: 2K floats (h2 then h1)")
             w = weights.ctypes.data_as(C.POINTER(C.c_float))
         self._check(_lib.easgd_exchange(self._h, m, w, alpha), "easgd_exchange")
+
+    def dw_order_next(self, seed, round_):
+        order = np.empty(self.K, np.uint16)
+        self._check(_lib.dw_order_next(self._h, int(seed), int(round_),
+                                       order.ctypes.data_as(C.POINTER(C.c_uint16))), "dw_order_next")
+        return order
+
+    def easgd_exchange_async(self, worker_mask=None, weights=None, alpha=0.0, order=None):
+        m = w = o = None
+        if worker_mask is not None:
+            worker_mask = np.ascontiguousarray(worker_mask, np.uint8)
+            m = worker_mask.ctypes.data_as(C.POINTER(C.c_uint8))
+        if weights is not None:
+            weights = np.ascontiguousarray(weights, np.float32)
+            if weights.size != 2 * self.K:
+                raise ValueError("weights: 2K floats (h2 then h1)")
+            w = weights.ctypes.data_as(C.POINTER(C.c_float))
+        if order is not None:
+            order = np.ascontiguousarray(order, np.uint16)
+            if order.size != self.K:
+                raise ValueError("order: K entries")
+            o = order.ctypes.data_as(C.POINTER(C.c_uint16))
+        self._check(_lib.easgd_exchange_async(self._h, m, w, alpha, o), "easgd_exchange_async")
 
     def ah_launch_count(self):
         return int(_lib.ah_launch_count(self._h))

@@ -8,50 +8,9 @@
 #include <new>
 #include <vector>
 
-#include "ah_internal.h"
+#include "ah_ctx.h"
 
 using namespace ah;
-
-struct ah_ctx {
-    int K = 0;
-    uint32_t P = 0;
-    uint64_t lds = 0;              // row stride of x, m, v, c (P rounded up to 4)
-    uint32_t ntiles = 0, ntiles_pad = 0;
-    int device = 0;
-    int sm_count = 0;
-    bool has_device = true;        // false: bookkeeping-only handle (AH_DEVICE_NONE)
-    std::vector<Run> runs_host;
-    std::vector<TileInfo> tiles_host;
-    cudaStream_t stream = nullptr;
-    bool owns_workspace = false;
-    void *workspace = nullptr;
-    size_t workspace_bytes = 0;
-
-    // device views into the workspace
-    float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
-    double *partials = nullptr, *scratch = nullptr;
-    double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
-    Run *runs = nullptr;
-    TileInfo *tiles = nullptr;
-    uint32_t nruns = 0;
-
-    // host state
-    double *norm2_host = nullptr;  // pinned copy of norm2_dev (status word + K doubles)
-    cudaEvent_t norm2_ready = nullptr;
-    bool norm2_pending = false;    // a want_dist step has been enqueued since the last read
-    double norm2_last[AH_MAX_WORKERS];
-    uint32_t step[AH_MAX_WORKERS];
-    uint32_t down_until[AH_MAX_WORKERS];
-    uint32_t calls = 0;            // ah_local_step calls so far
-    int p_hist = 4;
-    double coef[AH_MAX_HIST];
-    double kappa = -0.1;
-    std::vector<double> uhist;     // [K][p_hist + 1], newest first
-    int ring_filled = 0;
-
-    int last_cuda = 0;
-    uint64_t launches = 0;
-};
 
 namespace {
 

@@ -6,6 +6,7 @@ import numpy as np
 
 Z_SEED = 0x5EED0001
 MASK_SEED = 0x5EED0002
+ORDER_SEED = 0x5EED0003
 
 
 @dataclass
@@ -26,6 +27,7 @@ class RunConfig:
     weight_decay: float = 0.0
     alpha: float | None = None      # None: min(0.05, 0.8 / K)
     dynamic: bool = True            # dynamic weights (else fixed alpha)
+    asynchronous: bool = False      # workers reach the master one at a time, seeded order
     scripted: list = field(default_factory=list)
     pool: int = 3
     data_seed: int = 0
@@ -54,7 +56,8 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
     h.ah_broadcast_center()
     ref = oracle_mod.OracleState(theta0, cfg.K, cfg.segments, variant=variant)
     alpha = cfg.alpha_value()
-    log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "exchanges": 0}
+    log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "orders_equal": True,
+           "exchanges": 0}
     for t in range(1, cfg.rounds + 1):
         mask_g = h.dw_mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
         mask_o = ref.mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
@@ -72,17 +75,22 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                        active=mask_o if cfg.frozen else None, **common)
         if ex:
             log["exchanges"] += 1
+            w = h2 = h1 = None
             if cfg.dynamic:
                 w = h.dw_weights_next(alpha)
                 h2, h1 = ref.weights_next(alpha)
                 log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
                 log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], h2) and
                                              np.array_equal(w[cfg.K:], h1))
-                h.easgd_exchange(mask_g, w, alpha)
-                ref.exchange(mask_o, h2, h1)
+            if cfg.asynchronous:
+                order_g = h.dw_order_next(ORDER_SEED, t)
+                order_o = ref.order_next(ORDER_SEED, t)
+                log["orders_equal"] &= bool(np.array_equal(order_g, order_o))
+                h.easgd_exchange_async(mask_g, w, alpha, order_g)
+                ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
             else:
-                h.easgd_exchange(mask_g, None, alpha)
-                ref.exchange(mask_o, alpha=alpha)
+                h.easgd_exchange(mask_g, w, alpha)
+                ref.exchange(mask_o, h2, h1, alpha=alpha)
         if check_every and t % check_every == 0:
             assert tolerance_violations(h.ah_state_get(binding.AH_X), ref.x) == 0, t
     return h, ref, log

@@ -172,6 +172,63 @@ def test_exchange_alpha_zero_is_identity(B, torch):
     h.close()
 
 
+# --------------------------------------------------- asynchronous exchange
+@pytest.mark.parametrize("K,P", [(1, 7), (3, 1000), (4, 4099), (7, 2048), (16, 10_001), (64, 3001),
+                                 (256, 1030)])
+def test_exchange_async_bit_exact(B, torch, K, P):
+    rng = np.random.default_rng(K * 1000 + P + 1)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    x = theta0[None] + rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.05)
+    h = B.Handle(K, P, [])
+    ref = OracleState(theta0, K, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x)
+    ref.x[:] = x
+    for trial in range(5):
+        mask = (rng.random(K) > 0.3).astype(np.uint8) if trial else None
+        if trial == 3:
+            mask[:] = 0                                    # nobody arrives
+        order = None if trial == 4 else h.dw_order_next(77, trial)
+        if trial != 4:
+            assert np.array_equal(order, ref.order_next(77, trial))
+        if trial % 2 == 0:
+            h2 = rng.uniform(0, 0.3, K).astype(np.float32)   # sum far above 1: fine when sequential
+            h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+            h.easgd_exchange_async(mask, np.concatenate([h2, h1]), 0.0, order)
+            ref.exchange_async(mask, h2, h1, order=order)
+        else:
+            h.easgd_exchange_async(mask, None, 0.25, order)
+            ref.exchange_async(mask, alpha=0.25, order=order)
+        assert np.array_equal(h.ah_state_get(B.AH_X), ref.x), trial
+        assert np.array_equal(h.ah_state_get(B.AH_CENTER), ref.center), trial
+    # an order that is not a permutation is refused and nothing moves
+    if K > 1:
+        bad = np.arange(K, dtype=np.uint16)
+        bad[0] = bad[1]
+        with pytest.raises(B.AdaHessError) as e:
+            h.easgd_exchange_async(None, None, 0.1, bad)
+        assert e.value.status == B.AH_ERR_INVALID_ARG
+        bad[0] = K
+        with pytest.raises(B.AdaHessError):
+            h.easgd_exchange_async(None, None, 0.1, bad)
+        assert np.array_equal(h.ah_state_get(B.AH_X), ref.x)
+    h.close()
+
+
+def test_async_rounds_resnet18_shape_reduced(B, torch):
+    # the whole round with the asynchronous exchange: dynamic weights, Bernoulli(1/3)
+    # communication failures (Sec. VI), seeded arrival order, alpha = 0.1 (Sec. VII) for
+    # K = 8, where the simultaneous form would sit at its stability limit
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=120, tau=2,
+                    p_fail=1 / 3, alpha=0.1, asynchronous=True)
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"] and log["orders_equal"]
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    h.close()
+
+
 # ---------------------------------------------------- whole configurations
 def _check_run(B, cfg, inputs, bit_exact=True):
     h, ref, log = run_gaussian(cfg, B, oracle, inputs, variant="omp")

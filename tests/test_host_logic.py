@@ -67,6 +67,7 @@ def test_bookkeeping_handle_refuses_device_calls(B):
     h = B.Handle(2, 64, [(0, 64, 1)], host_only=True)
     assert B.raw().ah_broadcast_center(h._h) == B.AH_ERR_STATE
     assert B.raw().easgd_exchange(h._h, None, None, 0.1) == B.AH_ERR_STATE
+    assert B.raw().easgd_exchange_async(h._h, None, None, 0.1, None) == B.AH_ERR_STATE
     w = (C.c_float * 4)()
     assert B.raw().dw_weights_next(h._h, 0.1, w) == B.AH_ERR_STATE
     h.close()
@@ -80,6 +81,17 @@ def test_mask_matches_oracle_bit_for_bit(B):
             assert np.array_equal(h.dw_mask_next(0x5EED0002, t, p, stale),
                                   ref.mask_next(0x5EED0002, t, p, stale)), (K, p, stale, t)
         assert np.array_equal(h.ah_state_get(B.AH_DOWN_UNTIL), ref.down_until)
+        h.close()
+
+
+def test_arrival_order_matches_oracle_bit_for_bit(B):
+    for K in (1, 2, 3, 8, 64, 256):
+        h = B.Handle(K, 8, [], host_only=True)
+        ref = OracleState(np.zeros(8, np.float32), K, [])
+        for t in (0, 1, 2, 3, 1000, 0xFFFFFFFE):
+            for seed in (0x5EED0003, 0xFEDCBA9876543210):
+                got = h.dw_order_next(seed, t)
+                assert got.dtype == np.uint16 and np.array_equal(got, ref.order_next(seed, t)), (K, t)
         h.close()
 
 
