@@ -97,32 +97,54 @@ __device__ __forceinline__ void consumer_sync()
 // x / b for a divisor b whose correctly rounded reciprocal r is known: one
 // multiply, the exact remainder by FMA, one correction (Markstein's sequence).  The
 // result is the correctly rounded quotient whenever no intermediate leaves the
-// normal range, which the exponent test guarantees for 2^-24 < b <= 1; outside that
-// window of x the plain division is used.  (Checked exhaustively on the host, for
-// every x in the window, against several hundred divisors of the form 1 - beta^t.)
+// normal range, which holds for 2^-24 < b <= 128 when 2^-63 <= |x| < 2^64 (checked
+// exhaustively on the host for every significand of x, for the integer divisors
+// 2..128 and for divisors of the form 1 - beta^t).  Callers test the window.
+__device__ __forceinline__ float div_by_const_in_window(float x, float b, float r)
+{
+    const float q = __fmul_rn(x, r);
+    const float rem = __fmaf_rn(-b, q, x);
+    return __fmaf_rn(rem, r, q);
+}
+
+__device__ __forceinline__ bool in_window(float lo_abs, float hi_abs)
+{
+    return lo_abs >= 0x1p-63f && hi_abs < 0x1p64f;
+}
+
 __device__ __forceinline__ float div_by_const(float x, float b, float r)
 {
-    const uint32_t e = (__float_as_uint(x) >> 23) & 0xffu;
-    if (e - 64u < 127u) {
-        const float q = __fmul_rn(x, r);
-        const float rem = __fmaf_rn(-b, q, x);
-        return __fmaf_rn(rem, r, q);
-    }
-    return __fdiv_rn(x, b);
+    const float a = fabsf(x);
+    return in_window(a, a) ? div_by_const_in_window(x, b, r) : __fdiv_rn(x, b);
+}
+
+__device__ __forceinline__ float min_abs4(float4 a)
+{
+    return fminf(fminf(fabsf(a.x), fabsf(a.y)), fminf(fabsf(a.z), fabsf(a.w)));
+}
+
+__device__ __forceinline__ float max_abs4(float4 a)
+{
+    return fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w)));
 }
 
 // Per-element AdaHessian update (Sec. IV-B of the paper; Eq. 4 with the diagonal
-// preconditioner 1 / ((sqrt vhat)^k + eps)).  D is the spatially averaged
-// Hutchinson estimate of the Hessian diagonal for this element.
+// preconditioner 1 / ((sqrt vhat)^k + eps)), split in two so that four elements can
+// share one test of the division window.  D is the spatially averaged Hutchinson
+// estimate of the Hessian diagonal for this element.
 // POWMODE: 0 -> k = 1, 1 -> k = 1/2, 2 -> general k via powf.
-template <int POWMODE, bool WD>
-__device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, float g, float D,
-                                                  const StepParams &p, const WorkerConst &w)
+__device__ __forceinline__ void moments(float &m, float &v, float g, float D, const StepParams &p)
 {
-    const float m1 = __fadd_rn(__fmul_rn(p.beta1, m), __fmul_rn(p.omb1, g));
-    const float v1 = __fadd_rn(__fmul_rn(p.beta2, v), __fmul_rn(__fmul_rn(p.omb2, D), D));
-    const float mhat = div_by_const(m1, w.bc1, w.rbc1);
-    const float vhat = div_by_const(v1, w.bc2, w.rbc2);
+    m = __fadd_rn(__fmul_rn(p.beta1, m), __fmul_rn(p.omb1, g));
+    v = __fadd_rn(__fmul_rn(p.beta2, v), __fmul_rn(__fmul_rn(p.omb2, D), D));
+}
+
+template <int POWMODE, bool WD, bool WINDOW>
+__device__ __forceinline__ float step_from_moments(float x, float m1, float v1, const StepParams &p,
+                                                   const WorkerConst &w)
+{
+    const float mhat = WINDOW ? div_by_const_in_window(m1, w.bc1, w.rbc1) : __fdiv_rn(m1, w.bc1);
+    const float vhat = WINDOW ? div_by_const_in_window(v1, w.bc2, w.rbc2) : __fdiv_rn(v1, w.bc2);
     const float r = __fsqrt_rn(vhat);
     float pw;
     if (POWMODE == 0) pw = r;
@@ -130,24 +152,58 @@ __device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, 
     else pw = powf(r, p.hpow);
     const float den = __fadd_rn(pw, p.eps);
     const float q = __fdiv_rn(mhat, den);
-    float xn;
-    if (WD) xn = __fsub_rn(x, __fmul_rn(p.lr, __fadd_rn(q, __fmul_rn(p.wd, x))));
-    else    xn = __fsub_rn(x, __fmul_rn(p.lr, q));
-    x = xn; m = m1; v = v1;
+    if (WD) return __fsub_rn(x, __fmul_rn(p.lr, __fadd_rn(q, __fmul_rn(p.wd, x))));
+    return __fsub_rn(x, __fmul_rn(p.lr, q));
 }
 
-__device__ __forceinline__ float flip_if(float a, uint32_t bit)
+template <int POWMODE, bool WD>
+__device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, float g, float D,
+                                                  const StepParams &p, const WorkerConst &w)
 {
-    return __uint_as_float(__float_as_uint(a) ^ (bit << 31));
+    moments(m, v, g, D, p);
+    const float lo = fminf(fabsf(m), fabsf(v)), hi = fmaxf(fabsf(m), fabsf(v));
+    x = in_window(lo, hi) ? step_from_moments<POWMODE, WD, true>(x, m, v, p, w)
+                          : step_from_moments<POWMODE, WD, false>(x, m, v, p, w);
+}
+
+// Four consecutive elements at once: one window test for the eight divisions.
+template <int POWMODE, bool WD>
+__device__ __forceinline__ void adahessian_update4(float4 &x, float4 &m, float4 &v, const float4 g,
+                                                   const float4 D, const StepParams &p,
+                                                   const WorkerConst &w)
+{
+    moments(m.x, v.x, g.x, D.x, p);
+    moments(m.y, v.y, g.y, D.y, p);
+    moments(m.z, v.z, g.z, D.z, p);
+    moments(m.w, v.w, g.w, D.w, p);
+    const float lo = fminf(min_abs4(m), min_abs4(v)), hi = fmaxf(max_abs4(m), max_abs4(v));
+    if (in_window(lo, hi)) {
+        x.x = step_from_moments<POWMODE, WD, true>(x.x, m.x, v.x, p, w);
+        x.y = step_from_moments<POWMODE, WD, true>(x.y, m.y, v.y, p, w);
+        x.z = step_from_moments<POWMODE, WD, true>(x.z, m.z, v.z, p, w);
+        x.w = step_from_moments<POWMODE, WD, true>(x.w, m.w, v.w, p, w);
+    } else {
+        x.x = step_from_moments<POWMODE, WD, false>(x.x, m.x, v.x, p, w);
+        x.y = step_from_moments<POWMODE, WD, false>(x.y, m.y, v.y, p, w);
+        x.z = step_from_moments<POWMODE, WD, false>(x.z, m.z, v.z, p, w);
+        x.w = step_from_moments<POWMODE, WD, false>(x.w, m.w, v.w, p, w);
+    }
+}
+
+// a with its sign flipped when bit K of bits is set.
+template <int K>
+__device__ __forceinline__ float flip_if_bit(float a, uint32_t bits)
+{
+    return __uint_as_float(__float_as_uint(a) ^ ((bits << (31 - K)) & 0x80000000u));
 }
 
 // z (.) h for four consecutive elements; bit k of nib set means z = -1 for lane k.
 __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 {
-    h.x = flip_if(h.x, nib & 1u);
-    h.y = flip_if(h.y, (nib >> 1) & 1u);
-    h.z = flip_if(h.z, (nib >> 2) & 1u);
-    h.w = flip_if(h.w, (nib >> 3) & 1u);
+    h.x = flip_if_bit<0>(h.x, nib);
+    h.y = flip_if_bit<1>(h.y, nib);
+    h.z = flip_if_bit<2>(h.z, nib);
+    h.w = flip_if_bit<3>(h.w, nib);
     return h;
 }
 
@@ -228,12 +284,13 @@ struct __align__(128) Shared {
 template <int B>
 __device__ __forceinline__ void block_means_fixed(float *base, uint32_t nblk, int ctid)
 {
+    const float fb = (float)B, rb = __frcp_rn(fb);
     for (uint32_t k = ctid; k < nblk; k += kConsumers) {
         float *blk = base + k * B;
         float S = blk[0];
 #pragma unroll
         for (int e = 1; e < B; ++e) S = __fadd_rn(S, blk[e]);
-        const float mean = __fdiv_rn(S, (float)B);
+        const float mean = div_by_const(S, fb, rb);
 #pragma unroll
         for (int e = 0; e < B; ++e) blk[e] = mean;
     }
@@ -241,12 +298,12 @@ __device__ __forceinline__ void block_means_fixed(float *base, uint32_t nblk, in
 
 __device__ __forceinline__ void block_means_any(float *base, uint32_t nblk, uint32_t B, int ctid)
 {
-    const float fb = (float)B;
+    const float fb = (float)B, rb = __frcp_rn(fb);
     for (uint32_t k = ctid; k < nblk; k += kConsumers) {
         float *blk = base + k * B;
         float S = blk[0];
         for (uint32_t e = 1; e < B; ++e) S = __fadd_rn(S, blk[e]);
-        const float mean = __fdiv_rn(S, fb);
+        const float mean = div_by_const(S, fb, rb);
         for (uint32_t e = 0; e < B; ++e) blk[e] = mean;
     }
 }
@@ -374,10 +431,13 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     }
                     const float4 g = ld_vec(&st.g[off]);
                     float4 x = ld_vec(&st.x[off]), m = ld_vec(&st.m[off]), v = ld_vec(&st.v[off]);
-                    adahessian_update<POWMODE, WD>(x.x, m.x, v.x, g.x, D.x, p, w);
-                    if (nv > 1) adahessian_update<POWMODE, WD>(x.y, m.y, v.y, g.y, D.y, p, w);
-                    if (nv > 2) adahessian_update<POWMODE, WD>(x.z, m.z, v.z, g.z, D.z, p, w);
-                    if (nv > 3) adahessian_update<POWMODE, WD>(x.w, m.w, v.w, g.w, D.w, p, w);
+                    if (nv == 4) {
+                        adahessian_update4<POWMODE, WD>(x, m, v, g, D, p, w);
+                    } else {     // ragged end of the row: lanes past P keep their (zero) state
+                        adahessian_update<POWMODE, WD>(x.x, m.x, v.x, g.x, D.x, p, w);
+                        if (nv > 1) adahessian_update<POWMODE, WD>(x.y, m.y, v.y, g.y, D.y, p, w);
+                        if (nv > 2) adahessian_update<POWMODE, WD>(x.z, m.z, v.z, g.z, D.z, p, w);
+                    }
                     st_vec(xr + off, x);
                     st_vec(mr + off, m);
                     st_vec(vr + off, v);

@@ -149,3 +149,17 @@ def test_tile_descriptors_cover_whole_blocks(B, name):
             s, e, b, _ = (int(v) for v in runs[r])
             assert (edge - s) % b == 0 or edge == e
     h.close()
+
+
+def test_constant_divisor_shortcut_is_exact(tmp_path):
+    # the kernels divide by per-launch constants (bias corrections, spatial block sizes)
+    # with a reciprocal multiply plus one FMA correction; a C program checks on the host,
+    # for every binary32 significand, that this equals the correctly rounded quotient
+    import subprocess
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "helpers", "exact_division_check.c")
+    exe = str(tmp_path / "exact_division_check")
+    subprocess.check_call(["gcc", "-O2", "-mfma", "-ffp-contract=off", "-fopenmp", src, "-o", exe, "-lm"])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout
+    checked, bad = (int(v) for v in out.stdout.split()[1::2])
+    assert checked > 200 and bad == 0
