@@ -113,6 +113,9 @@ class Oracle:
         L.orc_exchange_async.restype = None
         L.orc_order_next.argtypes = [C.c_int, C.c_uint64, C.c_uint32, pu16]
         L.orc_order_next.restype = None
+        L.orc_sgd_step.argtypes = [pf, pf, pu32, pf, C.c_int, C.c_uint64, C.c_uint64, C.c_float,
+                                   C.c_float, pu8]
+        L.orc_sgd_step.restype = None
         L.orc_is_double.restype = C.c_int
         L.orc_num_threads.restype = C.c_int
 
@@ -232,6 +235,17 @@ class OracleState:
             lr, beta1, beta2, eps, hessian_power, weight_decay, _u8(active))
         if rc != 0:
             raise MemoryError("oracle scratch allocation failed")
+        if want_dist:
+            self.norm2 = self.o.norm2(self.x, self.center)
+
+    # first-order local steps (EASGD / EAMSGD): the velocity lives in self.m
+    def sgd_step(self, grad, lr, momentum=0.0, active=None, want_dist=False):
+        assert grad.dtype == np.float32 and grad.shape[0] == self.K and grad.flags.c_contiguous
+        if active is not None:
+            active = np.ascontiguousarray(active, np.uint8)
+        self.o.lib.orc_sgd_step(_f32(self.x), _f32(self.m),
+                                self.step.ctypes.data_as(C.POINTER(C.c_uint32)), _f32(grad),
+                                self.K, self.P, grad.shape[1], lr, momentum, _u8(active))
         if want_dist:
             self.norm2 = self.o.norm2(self.x, self.center)
 

@@ -430,6 +430,38 @@ void orc_order_next(int K, uint64_t seed, uint32_t t, uint16_t *order)
     }
 }
 
+/* ------------------------------------------------------------------------- */
+/* First-order local steps of the methods the paper compares against (Sec. VI:
+ * EASGD and EAMSGD, "EASGD with Momentum"; Sec. VII: eta = 0.01, delta = 0.5).
+ *   plain SGD (Eqs. 2-3, momentum == 0):   x <- x - (eta g)
+ *   momentum delta (velocity form):        u <- (delta u) - (eta g);   x <- x + u
+ * u[K][P] is the velocity (the paper does not print the momentum rule; this is the
+ * classical form of the works it cites for it; with Nesterov's variant only the point
+ * where the caller evaluates g changes).  Inactive workers are left untouched; an
+ * active worker's step count goes up by one.                                     */
+/* ------------------------------------------------------------------------- */
+void orc_sgd_step(float *x, float *u, uint32_t *step, const float *grad, int K, uint64_t P,
+                  uint64_t ld, float lr, float momentum, const uint8_t *active)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int i = 0; i < K; ++i) {
+        if (active && !active[i]) continue;
+        step[i] += 1;
+        const real eta = (real)lr, delta = (real)momentum;
+        const float *g = grad + (uint64_t)i * ld;
+        float *xi = x + (uint64_t)i * P, *ui = u + (uint64_t)i * P;
+        for (uint64_t j = 0; j < P; ++j) {
+            if (momentum == 0.0f) {
+                xi[j] = (float)((real)xi[j] - (eta * (real)g[j]));
+            } else {
+                const real un = (delta * (real)ui[j]) - (eta * (real)g[j]);
+                ui[j] = (float)un;
+                xi[j] = (float)((real)xi[j] + (real)(float)un);
+            }
+        }
+    }
+}
+
 int orc_is_double(void)
 {
 #ifdef ORC_DOUBLE
