@@ -47,6 +47,7 @@ WORKLOADS = {
     "p18k4": ("resnet18", 4, 4, 0.1, 1, False),
     "pvggk1": ("vgg16", 1, 4, 0.1, 1, False),
 }
+SGD_LR, SGD_MOMENTUM = 0.01, 0.5          # Sec. VII: eta = 0.01, delta = 0.5
 HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weight_decay=0.0)
 
 # DRAM bytes per parameter update of the fused local-step kernel, from one ncu capture
@@ -129,7 +130,8 @@ class ClockSampler:
                 "samples": len(clocks), "reasons": sorted(reasons)}
 
 
-def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None):
+def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
+               method="adahessian"):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
     memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
@@ -146,21 +148,27 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
             host_pool, g, hv = stage
             hg, hh = host_pool[t % len(host_pool)]
             g.copy_(hg, non_blocking=True)
-            hv.copy_(hh, non_blocking=True)
+            if method == "adahessian":
+                hv.copy_(hh, non_blocking=True)
         else:
             g, hv = pool[t % len(pool)]
         if events is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-        h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
-                        **HYPER)
+        first_order = method != "adahessian"     # EASGD / EAMSGD: fixed alpha, no distances
+        if first_order:
+            h.sgd_local_step(g, SGD_LR, SGD_MOMENTUM if method == "msgd" else 0.0,
+                             active=mask if frozen else None)
+        else:
+            h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
+                            **HYPER)
         n_act = int(mask.sum()) if frozen else K
         worker_steps += n_act
         if events is not None:
             e1.record()
             events.append((e0, e1, ex, n_act))
         if ex:
-            w = h.dw_weights_next(alpha)
+            w = None if first_order else h.dw_weights_next(alpha)
             if ex_events is not None:
                 x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 x0.record()
@@ -214,7 +222,7 @@ def gpu_arm(args):
     t = 0
     asyn = args.exchange == "async"
     for _ in range(args.warmup):
-        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn)
+        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -225,7 +233,8 @@ def gpu_arm(args):
     start.record()
     worker_steps = exchanged = 0
     for _ in range(args.steps):
-        t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events)
+        t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events,
+                                method=args.method)
         worker_steps += ws
         exchanged += exd
     stop.record()
@@ -247,7 +256,11 @@ def gpu_arm(args):
     withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex]
     # algorithmic bytes of a launch: 32 per update; a distance round also reads the
     # master row once and the x of every worker that sat the step out
-    if plain:
+    bpu = {"adahessian": 32, "sgd": 12, "msgd": 20}[args.method]
+    if args.method != "adahessian":
+        dom, dom_name = plain + withd, "sgd_step"       # no distance rounds with a fixed alpha
+        dom_bytes = sum(bpu * P * n for _, n in dom) / len(dom)
+    elif plain:
         dom, dom_name = plain, "local_step"
         dom_bytes = sum(32 * P * n for _, n in dom) / len(dom)
     else:
@@ -257,7 +270,8 @@ def gpu_arm(args):
     peak, peak_kind = measured_hbm_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["sources_sha256"] == kernel_sources_hash() and NCU_TRAFFIC["dram_bytes_per_update"]:
+    if (args.method == "adahessian" and NCU_TRAFFIC["sources_sha256"] == kernel_sources_hash()
+            and NCU_TRAFFIC["dram_bytes_per_update"]):
         traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
@@ -265,7 +279,7 @@ def gpu_arm(args):
                 "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
                 "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
-    run_bytes = 32 * P * worker_steps + 8 * P * exchanged + 12 * P * args.steps
+    run_bytes = bpu * P * worker_steps + 8 * P * exchanged + (12 if bpu == 32 else 8) * P * args.steps
     whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
     # the exchange kernel alone: 8 bytes per (arriving worker, parameter) + 8 per parameter
@@ -286,12 +300,14 @@ def gpu_arm(args):
         host_pool = [(g.cpu().pin_memory(), hv.cpu().pin_memory()) for g, hv in pool[:n_host]]
         sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
-        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn)
+        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn,
+                             method=args.method)
         barrier()
         start.record()
         e2e_ws = 0
         for _ in range(e2e_steps):
-            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn)
+            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn,
+                                  method=args.method)
             e2e_ws += ws
         stop.record()
         barrier()
@@ -302,7 +318,8 @@ def gpu_arm(args):
             ems = float(tmax.item())
         e2e = {"value": round(e2e_ws * P * world / (ems * 1e-3) / 1e9, 3),
                "unit": "G param-updates/s", "steps": e2e_steps,
-               "h2d_bytes_per_step": pair_bytes * tau, "d2h_bytes_per_step": 8 * K}
+               "h2d_bytes_per_step": (pair_bytes if bpu == 32 else pair_bytes // 2) * tau,
+               "d2h_bytes_per_step": 8 * K if bpu == 32 else 0}
 
     out = {
         "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
@@ -314,6 +331,9 @@ def gpu_arm(args):
                                f"p_fail={p_fail}, max_stale={max_stale}, frozen_stragglers={frozen}",
                    "step": f"one communication period = {tau} rounds + 1 exchange",
                    "exchange": "asynchronous, seeded arrival order" if asyn else "simultaneous",
+                   "local_step": {"adahessian": "AdaHessian, dynamic weights",
+                                  "sgd": "SGD, fixed alpha (EASGD)",
+                                  "msgd": "SGD with momentum 0.5, fixed alpha (EAMSGD)"}[args.method],
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
                    "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
@@ -375,13 +395,17 @@ def oracle_periods(args, layout, periods, warm):
                 worker_steps += int(mask.sum()) if frozen else K
             ex = r == tau - 1
             g, hv = pool[t % 2]
-            st.local_step(g, hv, Z_SEED, t, active=mask if frozen else None, want_dist=ex, **HYPER)
+            if args.method == "adahessian":
+                st.local_step(g, hv, Z_SEED, t, active=mask if frozen else None, want_dist=ex, **HYPER)
+            else:
+                st.sgd_step(g, SGD_LR, SGD_MOMENTUM if args.method == "msgd" else 0.0,
+                            active=mask if frozen else None)
             if ex:
-                h2, h1 = st.weights_next(alpha)
+                h2, h1 = st.weights_next(alpha) if args.method == "adahessian" else (None, None)
                 if args.exchange == "async":
-                    st.exchange_async(mask, h2, h1, order=st.order_next(ORDER_SEED, t))
+                    st.exchange_async(mask, h2, h1, alpha=alpha, order=st.order_next(ORDER_SEED, t))
                 else:
-                    st.exchange(mask, h2, h1)
+                    st.exchange(mask, h2, h1, alpha=alpha)
     return time.perf_counter() - t_start, K, P, tau, min(threads, st.o.num_threads()), worker_steps
 
 
@@ -431,6 +455,8 @@ def main():
     ap.add_argument("--pool", type=int, default=4, help="grad/hvp pairs kept in HBM")
     ap.add_argument("--exchange", default="simultaneous", choices=["simultaneous", "async"],
                     help="all workers against the same master value, or one at a time")
+    ap.add_argument("--method", default="adahessian", choices=["adahessian", "sgd", "msgd"],
+                    help="local step: the paper's method, or the EASGD / EAMSGD comparison methods")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

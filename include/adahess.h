@@ -88,6 +88,14 @@ typedef struct {
                              K workers, into the handle (read by dw_weights_next)           */
 } ah_hyper;
 
+/* Hyper-parameters of one first-order local step (sgd_local_step). */
+typedef struct {
+    float lr;             /* eta                                                            */
+    float momentum;       /* delta in [0, 1); 0 = plain SGD, the velocity is not touched     */
+    const uint8_t *active;/* host pointer, K bytes, or NULL (all active), as in ah_hyper    */
+    int want_dist;        /* 1 = also compute ||x_i - c||^2 after the step, as in ah_hyper  */
+} sgd_hyper;
+
 /* Optional placement: caller-owned device memory and stream.  workspace must be
  * 256-byte aligned, at least ah_workspace_bytes() long, and outlive the handle; the
  * library never frees it.  With opt == NULL the handle allocates its own memory
@@ -182,6 +190,18 @@ int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
                   uint64_t z_seed, const ah_hyper *hy);
+
+/* One first-order local step of every active worker, the local optimiser of the
+ * EASGD and EAMSGD methods the paper compares against (Sec. VI; Sec. VII uses
+ * eta = 0.01, delta = 0.5):
+ *     momentum == 0 (Eqs. 2-3):   x = x - lr * grad
+ *     momentum  > 0:              u = momentum * u - lr * grad;   x = x + u
+ * The velocity u lives in the handle's first-moment rows (AH_M); the second-moment
+ * rows are not touched.  A handle should be driven by one kind of local step.  grad,
+ * ld, active, want_dist and the step counts behave as in ah_local_step; no Rademacher
+ * stream is consumed.  Memory traffic: 12 bytes per parameter update, 20 with momentum.
+ * Errors: INVALID_ARG, ALIGN, CUDA. */
+int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *hy);
 
 /* Parameters of the dynamic weighting rule (Sec. V-B): history depth p, the
  * coefficients c_0..c_{p-1} of Eqs. 10-11 (c_0 weighs the newest difference; they

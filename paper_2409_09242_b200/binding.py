@@ -35,7 +35,7 @@ AH_DEVICE_NONE = -2
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_local_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "ah_distances_static", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "sgd_local_step", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -48,6 +48,11 @@ class ah_hyper(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
                 ("eps", C.c_float), ("hessian_power", C.c_float), ("weight_decay", C.c_float),
                 ("round", C.c_uint32), ("active", C.POINTER(C.c_uint8)), ("want_dist", C.c_int)]
+
+
+class sgd_hyper(C.Structure):
+    _fields_ = [("lr", C.c_float), ("momentum", C.c_float), ("active", C.POINTER(C.c_uint8)),
+                ("want_dist", C.c_int)]
 
 
 class ah_alloc(C.Structure):
@@ -71,6 +76,7 @@ _lib.dw_weights_from_norm2.argtypes = [_vp, C.POINTER(C.c_double), C.c_float, C.
 _lib.dw_mask_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_double, C.c_int,
                               C.POINTER(C.c_uint8)]
 _lib.easgd_exchange.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float]
+_lib.sgd_local_step.argtypes = [_vp, _vp, C.c_uint64, C.POINTER(sgd_hyper)]
 _lib.dw_order_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.POINTER(C.c_uint16)]
 _lib.easgd_exchange_async.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
                                       C.POINTER(C.c_uint16)]
@@ -276,6 +282,18 @@ class Handle:
                       1 if want_dist else 0)
         self._check(_lib.ah_local_step(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
                                        grad.stride(0), int(z_seed), C.byref(hy)), "ah_local_step")
+
+    def sgd_local_step(self, grad, lr, momentum=0.0, active=None, want_dist=False):
+        act = None
+        if active is not None:
+            act = np.ascontiguousarray(active, np.uint8)
+            if act.size != self.K:
+                raise ValueError("active: K bytes")
+        hy = sgd_hyper(lr, momentum,
+                       act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None,
+                       1 if want_dist else 0)
+        self._check(_lib.sgd_local_step(self._h, _dev_ptr(grad, "grad"), grad.stride(0), C.byref(hy)),
+                    "sgd_local_step")
 
     def dw_config(self, p_hist, c, kappa):
         c = np.ascontiguousarray(c, np.float64)

@@ -54,3 +54,7 @@ inline int ah_cuda_fail(ah_ctx *h, cudaError_t e)
     if (h) h->last_cuda = (int)e;
     return AH_ERR_CUDA;
 }
+
+namespace ah {
+int finish_distances(ah_ctx *h);   // ah_host.cu
+}

@@ -129,6 +129,21 @@ void reset_history(ah_ctx *h)
 
 }  // namespace
 
+// After a step has left the tile partials of ||x_i - c||^2 in the workspace: finish
+// the pairwise tree on the device and start the copy of the K doubles (and the status
+// word in front of them) to pinned host memory.
+int ah::finish_distances(ah_ctx *h)
+{
+    AH_CUDA(h, launch_norm2_finalize(h->partials, h->scratch, h->ntiles, h->ntiles_pad, h->K,
+                                     h->norm2_dev + 1, h->stream));
+    h->launches += 1;
+    AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, (h->K + 1) * sizeof(double),
+                               cudaMemcpyDeviceToHost, h->stream));
+    AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
+    h->norm2_pending = true;
+    return AH_OK;
+}
+
 extern "C" {
 
 int ah_workspace_bytes(int K, uint64_t P, int nseg, size_t *out)
@@ -315,15 +330,7 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     p.nitems = p.nrows * h->ntiles;
     AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
     if (p.nitems) h->launches += 1;
-    if (dist) {
-        AH_CUDA(h, launch_norm2_finalize(h->partials, h->scratch, h->ntiles, h->ntiles_pad, h->K,
-                                         h->norm2_dev + 1, h->stream));
-        h->launches += 1;
-        AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, (h->K + 1) * sizeof(double),
-                                   cudaMemcpyDeviceToHost, h->stream));
-        AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
-        h->norm2_pending = true;
-    }
+    if (dist) return finish_distances(h);
     return AH_OK;
 }
 

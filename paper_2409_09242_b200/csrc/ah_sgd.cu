@@ -1,0 +1,140 @@
+// First-order local steps on the same batched [K, P] state: plain SGD (Eqs. 2-3 of
+// the paper) and SGD with momentum, the local optimisers of the EASGD and EAMSGD
+// methods the paper compares against (Sec. VI; eta = 0.01, delta = 0.5 in Sec. VII).
+// They share the exchange kernels and the distance / weight machinery with the
+// AdaHessian step.
+//
+// Pure streaming: 12 bytes per parameter update without momentum (read grad and x,
+// write x), 20 with it (the velocity is read and written too).  One CTA of 256
+// threads covers kTilesPerCta consecutive tiles of 1024 parameters of one worker,
+// one float4 per thread and tile, all loads issued before the first use.
+#include "ah_ctx.h"
+#include "ah_device.cuh"
+
+namespace ah {
+
+constexpr int kSgdThreads = 256;
+constexpr int kSgdTile = 1024;              // = kTile: a subtree of the distance tree
+#ifndef AH_SGD_TILES_PER_CTA
+#define AH_SGD_TILES_PER_CTA 4
+#endif
+constexpr int kTilesPerCta = AH_SGD_TILES_PER_CTA;
+static_assert(kSgdTile == kTile, "distance partials are indexed by the library's tile");
+
+struct SgdParams {
+    float *x, *u;                  // u: velocity (the handle's first-moment rows)
+    const float *c;
+    const float *grad;
+    double *partials;              // [K][ntiles_pad]
+    uint64_t lds, ld;
+    uint32_t P, ntiles, ntiles_pad;
+    float lr, momentum;
+    uint32_t nrows;
+    uint16_t row[AH_MAX_WORKERS];
+    uint8_t active[AH_MAX_WORKERS];
+};
+
+template <bool MOMENTUM, bool DIST>
+__global__ void __launch_bounds__(kSgdThreads)
+sgd_step_kernel(const __grid_constant__ SgdParams p)
+{
+    __shared__ double red[kTilesPerCta][kSgdThreads / 32];
+    const uint32_t i = p.row[blockIdx.y];
+    const bool act = p.active[i] != 0;
+    const uint32_t tile0 = blockIdx.x * (uint32_t)kTilesPerCta;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    float4 g[kTilesPerCta], x[kTilesPerCta], u[kTilesPerCta], c[kTilesPerCta];
+    uint32_t off[kTilesPerCta];
+#pragma unroll
+    for (int k = 0; k < kTilesPerCta; ++k) {
+        off[k] = (tile0 + k) * (uint32_t)kSgdTile + 4u * threadIdx.x;
+        if (off[k] < p.P) {
+            const uint64_t so = (uint64_t)i * p.lds + off[k];
+            x[k] = ld_vec(p.x + so);
+            if (act) g[k] = ld_vec(p.grad + (uint64_t)i * p.ld + off[k]);
+            if (MOMENTUM && act) u[k] = ld_vec(p.u + so);
+            if (DIST) c[k] = ld_vec(p.c + off[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kTilesPerCta; ++k) {
+        double d = 0.0;
+        if (off[k] < p.P) {
+            const int nv = p.P - off[k] >= 4u ? 4 : (int)(p.P - off[k]);
+            if (act) {
+                float *xe = &x[k].x, *ue = &u[k].x;
+                const float *ge = &g[k].x;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (e < nv) {            // lanes past P keep their zero state
+                        if (MOMENTUM) {
+                            ue[e] = __fsub_rn(__fmul_rn(p.momentum, ue[e]), __fmul_rn(p.lr, ge[e]));
+                            xe[e] = __fadd_rn(xe[e], ue[e]);
+                        } else {
+                            xe[e] = __fsub_rn(xe[e], __fmul_rn(p.lr, ge[e]));
+                        }
+                    }
+                }
+                const uint64_t so = (uint64_t)i * p.lds + off[k];
+                st_vec(p.x + so, x[k]);
+                if (MOMENTUM) st_vec(p.u + so, u[k]);
+            }
+            if (DIST) d = dist4(x[k], c[k], nv);
+        }
+        if (DIST) {
+            d = warp_tree_sum(d);
+            if (lane == 0) red[k][warp] = d;
+        }
+    }
+    if (DIST) {
+        __syncthreads();
+        if (threadIdx.x < kTilesPerCta && tile0 + threadIdx.x < p.ntiles)
+            p.partials[(uint64_t)i * p.ntiles_pad + tile0 + threadIdx.x] = tree8(red[threadIdx.x]);
+    }
+}
+
+template <bool MOMENTUM, bool DIST>
+static cudaError_t launch_sgd(const SgdParams &p, cudaStream_t s)
+{
+    const dim3 grid((p.ntiles + kTilesPerCta - 1) / kTilesPerCta, p.nrows);
+    if (p.nrows == 0) return cudaSuccess;
+    sgd_step_kernel<MOMENTUM, DIST><<<grid, kSgdThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace ah
+
+using namespace ah;
+
+extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *hy)
+{
+    if (!h || !grad || !hy || ld < h->P) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    if (!(hy->momentum >= 0.f && hy->momentum < 1.f)) return AH_ERR_INVALID_ARG;
+    if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0) return AH_ERR_ALIGN;
+
+    const bool dist = hy->want_dist != 0;
+    SgdParams p;
+    p.x = h->x; p.u = h->m; p.c = h->c; p.grad = grad;
+    p.partials = h->partials;
+    p.lds = h->lds; p.ld = ld;
+    p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
+    p.lr = hy->lr; p.momentum = hy->momentum;
+    p.nrows = 0;
+    for (int i = 0; i < h->K; ++i) {
+        const bool on = !hy->active || hy->active[i] != 0;
+        p.active[i] = on ? 1 : 0;
+        if (on) h->step[i] += 1;
+        if (on || dist) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
+    }
+    h->calls += 1;
+    cudaError_t e;
+    const bool mom = hy->momentum != 0.f;
+    if (mom) e = dist ? launch_sgd<true, true>(p, h->stream) : launch_sgd<true, false>(p, h->stream);
+    else     e = dist ? launch_sgd<false, true>(p, h->stream) : launch_sgd<false, false>(p, h->stream);
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    if (p.nrows) h->launches += 1;
+    if (dist) return finish_distances(h);
+    return AH_OK;
+}

@@ -28,6 +28,8 @@ class RunConfig:
     alpha: float | None = None      # None: min(0.05, 0.8 / K)
     dynamic: bool = True            # dynamic weights (else fixed alpha)
     asynchronous: bool = False      # workers reach the master one at a time, seeded order
+    method: str = "adahessian"      # local step: "adahessian", "sgd" or "msgd" (momentum)
+    momentum: float = 0.5
     scripted: list = field(default_factory=list)
     pool: int = 3
     data_seed: int = 0
@@ -69,10 +71,17 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         common = dict(lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
                       hessian_power=cfg.hessian_power, weight_decay=cfg.weight_decay,
                       want_dist=ex)
-        h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
-                        active=mask_g if cfg.frozen else None, **common)
-        ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
-                       active=mask_o if cfg.frozen else None, **common)
+        if cfg.method == "adahessian":
+            h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
+                            active=mask_g if cfg.frozen else None, **common)
+            ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
+                           active=mask_o if cfg.frozen else None, **common)
+        else:
+            delta = cfg.momentum if cfg.method == "msgd" else 0.0
+            h.sgd_local_step(dev_pool[k][0], cfg.lr, delta,
+                             active=mask_g if cfg.frozen else None, want_dist=ex)
+            ref.sgd_step(pool[k][0], cfg.lr, delta,
+                         active=mask_o if cfg.frozen else None, want_dist=ex)
         if ex:
             log["exchanges"] += 1
             w = h2 = h1 = None

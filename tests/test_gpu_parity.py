@@ -229,6 +229,59 @@ def test_async_rounds_resnet18_shape_reduced(B, torch):
     h.close()
 
 
+# ------------------------------------------- first-order local steps (EASGD / EAMSGD)
+@pytest.mark.parametrize("K,P", [(1, 1), (2, 1023), (3, 4097), (4, 184_837), (8, 4 * 1024 * 5), (5, 8193)])
+@pytest.mark.parametrize("delta", [0.0, 0.5])
+def test_sgd_step_bit_exact(B, torch, K, P, delta):
+    rng = np.random.default_rng(K * 7 + P)
+    ld = W.padded_ld(P) + 8
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    h = B.Handle(K, P, [])
+    ref = OracleState(theta0, K, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    for t in range(1, 7):
+        g = np.full((K, ld), np.nan, np.float32)             # columns past P must never be used
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32)
+        active = None if t % 3 else (rng.random(K) > 0.4).astype(np.uint8)
+        dist = t % 2 == 0
+        h.sgd_local_step(torch.from_numpy(g).cuda(), 0.01, delta, active=active, want_dist=dist)
+        ref.sgd_step(g, 0.01, delta, active=active, want_dist=dist)
+        if dist:
+            assert np.array_equal(h.ah_state_get(B.AH_NORM2), ref.norm2), t
+    assert np.array_equal(h.ah_state_get(B.AH_X), ref.x)
+    assert np.array_equal(h.ah_state_get(B.AH_M), ref.m)
+    assert not h.ah_state_get(B.AH_V).any()
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    h.close()
+
+
+@pytest.mark.parametrize("method,asyn", [("sgd", True), ("msgd", True), ("msgd", False)])
+def test_easgd_eamsgd_rounds_reduced(B, torch, method, asyn):
+    # the comparison methods of Sec. VI on the ResNet-18-shaped layout at 1/8 width: eta = 0.01,
+    # delta = 0.5, fixed alpha, communication suppressed one third of the time, tau = 2
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=4, segments=W.segments(layout), P=W.total_params(layout), rounds=90, tau=2,
+                    p_fail=1 / 3, alpha=0.1, dynamic=False, asynchronous=asyn, method=method)
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 4), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["orders_equal"]
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    h.close()
+
+
+def test_sgd_argument_checks(B, torch):
+    h = B.Handle(2, 100, [])
+    g = torch.zeros(2, 100, device="cuda")
+    with pytest.raises(B.AdaHessError) as e:
+        h.sgd_local_step(g, 0.1, 1.0)                        # momentum must stay below 1
+    assert e.value.status == B.AH_ERR_INVALID_ARG
+    with pytest.raises(B.AdaHessError) as e:
+        h.sgd_local_step(torch.zeros(2, 101, device="cuda")[:, 1:], 0.1)   # misaligned rows
+    assert e.value.status in (B.AH_ERR_ALIGN, B.AH_ERR_INVALID_ARG)
+    h.close()
+
+
 # ---------------------------------------------------- whole configurations
 def _check_run(B, cfg, inputs, bit_exact=True):
     h, ref, log = run_gaussian(cfg, B, oracle, inputs, variant="omp")

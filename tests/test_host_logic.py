@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol(B):
     for fn in os.listdir(os.path.join(root, "include")):
         text = open(os.path.join(root, "include", fn)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-        declared |= set(re.findall(r"\b((?:ah|dw|easgd)_[a-z0-9_]+)\s*\(", text))
+        declared |= set(re.findall(r"\b((?:ah|dw|easgd|sgd)_[a-z0-9_]+)\s*\(", text))
     assert {"ah_init", "ah_local_step", "easgd_exchange", "ah_state_get"} <= declared
     lib = C.CDLL(B._build.LIB_PATH)
     for name in sorted(declared):
