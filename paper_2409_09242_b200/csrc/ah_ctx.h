@@ -26,6 +26,7 @@ struct ah_ctx {
     float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
     double *partials = nullptr, *scratch = nullptr;
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
+    uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
     ah::Run *runs = nullptr;
     ah::TileInfo *tiles = nullptr;
     uint32_t nruns = 0;

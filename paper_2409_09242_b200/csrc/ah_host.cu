@@ -36,7 +36,7 @@ int cuda_fail(ah_ctx *h, cudaError_t e)
     } while (0)
 
 struct Layout {
-    size_t x, m, v, c, partials, scratch, norm2, runs, tiles, total;
+    size_t x, m, v, c, partials, scratch, norm2, sched, runs, tiles, total;
 };
 
 // Offsets of every array inside the workspace (each 256-byte aligned).
@@ -55,6 +55,7 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.partials = take((size_t)K * ntp * sizeof(double));
     L.scratch = take((size_t)K * ntp * sizeof(double));
     L.norm2 = take((size_t)(AH_MAX_WORKERS + 1) * sizeof(double));
+    L.sched = take(2 * sizeof(uint32_t));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
     L.total = off;
@@ -224,6 +225,7 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->partials = (double *)(base + L.partials);
     h->scratch = (double *)(base + L.scratch);
     h->norm2_dev = (double *)(base + L.norm2);
+    h->sched = (uint32_t *)(base + L.sched);
     h->runs = (Run *)(base + L.runs);
     h->tiles = (TileInfo *)(base + L.tiles);
 
@@ -301,6 +303,7 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     p.grad = grad; p.hvp = hvp;
     p.partials = h->partials;
     p.status = reinterpret_cast<uint32_t *>(h->norm2_dev);
+    p.sched = h->sched;
     p.runs = h->runs; p.tiles = h->tiles;
     p.lds = h->lds; p.ld = ld;
     p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;

@@ -81,6 +81,8 @@ struct StepParams {
     const float *grad, *hvp;
     double *partials;          // [K][ntiles_pad] tile sums of (x - c)^2
     uint32_t *status;          // device status word
+    uint32_t *sched;           // [0] next item to hand out, [1] producers that have left;
+                               // both zero between launches
     const Run *runs;
     const TileInfo *tiles;
     uint64_t lds;              // row stride of x, m, v (elements, multiple of 4)
