@@ -319,7 +319,11 @@ local_step_kernel(const __grid_constant__ StepParams p)
             }
             if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
             Stage<DIST> &st = sh.stage[s];
-            const uint32_t r = n / p.ntiles, tile = n - r * p.ntiles;
+            // Plain rounds walk one worker's row after the other; distance rounds walk
+            // the workers innermost, so that a tile of the master row is fetched from
+            // HBM once and served from L2 to the other workers.
+            const uint32_t tile = DIST ? n / p.nrows : n % p.ntiles;
+            const uint32_t r = DIST ? n - tile * p.nrows : n / p.ntiles;
             const uint32_t i = p.row[r];
             const bool act = p.active[i] != 0;
             const uint32_t t0 = tile * (uint32_t)kTile;
