@@ -116,6 +116,9 @@ class Oracle:
         L.orc_sgd_step.argtypes = [pf, pf, pu32, pf, C.c_int, C.c_uint64, C.c_uint64, C.c_float,
                                    C.c_float, pu8]
         L.orc_sgd_step.restype = None
+        L.orc_partition.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, pu32,
+                                    C.POINTER(C.c_uint64)]
+        L.orc_partition.restype = C.c_int
         L.orc_is_double.restype = C.c_int
         L.orc_num_threads.restype = C.c_int
 
@@ -173,6 +176,18 @@ class Oracle:
         order = np.empty(K, np.uint16)
         self.lib.orc_order_next(K, int(seed), int(t), order.ctypes.data_as(C.POINTER(C.c_uint16)))
         return order
+
+    def partition(self, seed, n, k, o):
+        """Data-overlap partition: (perm[n], bounds[k + 2]); O = perm[:o],
+        S_j = perm[bounds[j + 1]:bounds[j + 2]]."""
+        perm = np.empty(max(n, 1), np.uint32)
+        bounds = np.empty(k + 2, np.uint64)
+        rc = self.lib.orc_partition(int(seed), int(n), int(k), int(o),
+                                    perm.ctypes.data_as(C.POINTER(C.c_uint32)),
+                                    bounds.ctypes.data_as(C.POINTER(C.c_uint64)))
+        if rc != 0:
+            raise ValueError("partition: need o <= n and k >= 1")
+        return perm[:n], bounds
 
     def num_threads(self):
         return int(self.lib.orc_num_threads())

@@ -462,6 +462,40 @@ void orc_sgd_step(float *x, float *u, uint32_t *step, const float *grad, int K, 
     }
 }
 
+/* ------------------------------------------------------------------------- */
+/* Data overlap (Sec. V-A).  n data points, k workers, o shared points.  A seeded,
+ * uniformly random permutation perm of 0..n-1 is drawn (Fisher-Yates from the top:
+ * for q = n-1 down to 1, entries q and r mod (q+1) trade places, r = the 64-bit
+ * value (word1 << 32 | word0) of Philox(seed; (q low, q high, 0, 4))).  Then
+ *   O   = perm[0, o)                       the subset every worker receives
+ *   S_j = the next |S_j| entries, j = 0..k-1, dealt in order
+ *   D_j = O u S_j
+ * with |S_j| = floor((n-o)/k), plus one for the first (n-o) mod k workers so that
+ * the S_j cover D - O (the text states both; they agree when k divides n-o).
+ * bounds[0] = 0, bounds[1] = o, bounds[j+2] = end of S_j in perm.
+ * Returns 0, or -1 when o > n or k < 1.                                          */
+/* ------------------------------------------------------------------------- */
+int orc_partition(uint64_t seed, uint64_t n, uint32_t k, uint64_t o, uint32_t *perm, uint64_t *bounds)
+{
+    if (o > n || k < 1) return -1;
+    uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    for (uint64_t i = 0; i < n; ++i) perm[i] = (uint32_t)i;
+    for (uint64_t q = n; q-- > 1;) {
+        uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), 0u, 4u };
+        uint32_t r[4];
+        orc_philox4x32_10(ctr, key, r);
+        const uint64_t draw = ((uint64_t)r[1] << 32) | (uint64_t)r[0];
+        const uint64_t pick = draw % (q + 1);
+        const uint32_t tmp = perm[q]; perm[q] = perm[pick]; perm[pick] = tmp;
+    }
+    const uint64_t rest = n - o, base = rest / k, extra = rest % k;
+    bounds[0] = 0;
+    bounds[1] = o;
+    for (uint32_t j = 0; j < k; ++j)
+        bounds[j + 2] = bounds[j + 1] + base + (j < extra ? 1 : 0);
+    return 0;
+}
+
 int orc_is_double(void)
 {
 #ifdef ORC_DOUBLE
