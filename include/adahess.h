@@ -244,6 +244,22 @@ int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int ma
  * (h1_i = h2_i = alpha for all i).  alpha is ignored when weights != NULL. */
 int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha);
 
+/* ---- data overlap -------------------------------------------------------------- */
+
+/* Data-overlap partition (Sec. V-A): n data points, k workers; every worker receives
+ * the same `shared` points O plus its own disjoint subset S_j of the rest.
+ *   perm   : host pointer, n entries: a seeded uniformly random permutation of 0..n-1
+ *            (Fisher-Yates from the top; position q trades places with position
+ *            r mod (q+1), r = word1 << 32 | word0 of Philox4x32-10 with key
+ *            (seed low, seed high) and counter (q low, q high, 0, 4))
+ *   bounds : host pointer, k + 2 entries: O = perm[bounds[0], bounds[1]) with
+ *            bounds[0] = 0, bounds[1] = shared;  S_j = perm[bounds[j+1], bounds[j+2])
+ * |S_j| = floor((n - shared) / k), one more for the first (n - shared) mod k workers, so
+ * that the S_j cover everything outside O.  Worker j trains on O u S_j.
+ * Needs no handle and no GPU.  Errors: INVALID_ARG (shared > n, k < 1, n >= 2^32). */
+int dw_partition(uint64_t seed, uint64_t n, uint32_t k, uint64_t shared, uint32_t *perm,
+                 uint64_t *bounds);
+
 /* ---- asynchronous exchange ---------------------------------------------------- */
 
 /* Seeded arrival order for an asynchronous exchange round (Sec. II: training is

@@ -35,7 +35,7 @@ AH_DEVICE_NONE = -2
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_local_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "sgd_local_step", "ah_distances_static", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -77,6 +77,8 @@ _lib.dw_mask_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_double, C.c_int,
                               C.POINTER(C.c_uint8)]
 _lib.easgd_exchange.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float]
 _lib.sgd_local_step.argtypes = [_vp, _vp, C.c_uint64, C.POINTER(sgd_hyper)]
+_lib.dw_partition.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, C.POINTER(C.c_uint32),
+                              C.POINTER(C.c_uint64)]
 _lib.dw_order_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.POINTER(C.c_uint16)]
 _lib.easgd_exchange_async.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
                                       C.POINTER(C.c_uint16)]
@@ -138,6 +140,19 @@ def ah_distances_static(x, c, norm2_out, stream=None):
     if rc != AH_OK:
         raise AdaHessError(rc, "ah_distances_static")
     return norm2_out
+
+
+def dw_partition(seed, n, k, shared):
+    """Data-overlap partition: returns (perm[n] uint32, bounds[k + 2] uint64); the shared
+    subset is perm[:shared], worker j's own subset perm[bounds[j + 1]:bounds[j + 2]]."""
+    perm = np.empty(max(int(n), 1), np.uint32)
+    bounds = np.empty(int(k) + 2, np.uint64)
+    rc = _lib.dw_partition(int(seed), int(n), int(k), int(shared),
+                           perm.ctypes.data_as(C.POINTER(C.c_uint32)),
+                           bounds.ctypes.data_as(C.POINTER(C.c_uint64)))
+    if rc != AH_OK:
+        raise AdaHessError(rc, "dw_partition")
+    return perm[:int(n)], bounds
 
 
 def raw():

@@ -95,6 +95,18 @@ def test_arrival_order_matches_oracle_bit_for_bit(B):
         h.close()
 
 
+def test_partition_matches_oracle_bit_for_bit(B, orc):
+    for seed, n, k, o in ((0x5EED0004, 60000, 8, 7500), (1, 60000, 4, 15000), (2, 1000, 7, 0),
+                          (3, 17, 5, 3), (4, 10, 3, 10), (5, 1, 1, 0), (1 << 40 | 9, 4097, 16, 512)):
+        perm, bounds = B.dw_partition(seed, n, k, o)
+        rperm, rbounds = orc.partition(seed, n, k, o)
+        assert np.array_equal(perm, rperm) and np.array_equal(bounds, rbounds), (seed, n, k, o)
+    with pytest.raises(B.AdaHessError):
+        B.dw_partition(1, 10, 2, 11)
+    with pytest.raises(B.AdaHessError):
+        B.dw_partition(1, 10, 0, 1)
+
+
 def test_weights_match_oracle_bit_for_bit_given_same_distances(B):
     rng = np.random.default_rng(0)
     for K, alpha, p_hist, kappa in ((4, 0.05, 4, -0.1), (16, 0.1, 2, -0.05), (64, 0.0125, 6, -0.3)):
