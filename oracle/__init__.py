@@ -94,6 +94,14 @@ class Oracle:
                                      C.c_float, C.c_float, C.c_float, C.c_float, C.c_float,
                                      C.c_float, pu8]
         L.orc_local_step.restype = C.c_int
+        L.orc_local_step_n.argtypes = [pf, pf, pf, pu32, pf, pf, C.c_int, C.c_uint64, C.c_int,
+                                       C.c_uint64, C.c_uint64, ps, C.c_int, C.c_uint64, C.c_uint32,
+                                       C.c_float, C.c_float, C.c_float, C.c_float, C.c_float,
+                                       C.c_float, pu8]
+        L.orc_local_step_n.restype = C.c_int
+        L.orc_sample_z_s.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, C.c_uint64, pf,
+                                     C.c_uint64]
+        L.orc_sample_z_s.restype = None
         L.orc_norm2.argtypes = [pf, pf, C.c_int, C.c_uint64, pd]
         L.orc_norm2.restype = None
         L.orc_u_from_norm2.argtypes = [C.c_double]
@@ -133,6 +141,11 @@ class Oracle:
     def sample_z(self, seed, t, K, P):
         z = np.empty((K, P), np.float32)
         self.lib.orc_sample_z(seed, t, K, P, _f32(z), P)
+        return z
+
+    def sample_z_s(self, seed, t, sample, K, P):
+        z = np.empty((K, P), np.float32)
+        self.lib.orc_sample_z_s(seed, t, sample, K, P, _f32(z), P)
         return z
 
     def sample_zbits(self, seed, t, K, P):
@@ -238,15 +251,18 @@ class OracleState:
     # S2
     def local_step(self, grad, hvp, z_seed, t, lr, beta1=0.9, beta2=0.999, eps=1e-4,
                    hessian_power=1.0, weight_decay=0.0, active=None, want_dist=False):
+        """hvp: [K, ld] for one Hutchinson sample, or [n, K, ld] for n samples."""
         assert grad.dtype == np.float32 and hvp.dtype == np.float32
-        assert grad.shape[0] == self.K and grad.shape == hvp.shape and grad.flags.c_contiguous
+        assert grad.shape[0] == self.K and grad.flags.c_contiguous and hvp.flags.c_contiguous
         ld = grad.shape[1]
+        n = 1 if hvp.ndim == 2 else hvp.shape[0]
+        assert hvp.shape[-2:] == grad.shape
         if active is not None:
             active = np.ascontiguousarray(active, np.uint8)
-        rc = self.o.lib.orc_local_step(
+        rc = self.o.lib.orc_local_step_n(
             _f32(self.x), _f32(self.m), _f32(self.v),
             self.step.ctypes.data_as(C.POINTER(C.c_uint32)), _f32(grad), _f32(hvp),
-            self.K, self.P, ld, self._segs, len(self.segments), int(z_seed), int(t),
+            n, self.K * ld, self.K, self.P, ld, self._segs, len(self.segments), int(z_seed), int(t),
             lr, beta1, beta2, eps, hessian_power, weight_decay, _u8(active))
         if rc != 0:
             raise MemoryError("oracle scratch allocation failed")

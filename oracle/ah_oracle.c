@@ -82,7 +82,18 @@ enum { ORC_DOMAIN_Z = 0, ORC_DOMAIN_FAIL = 1, ORC_DOMAIN_STALE = 2 };
 /* Sign bit of the Rademacher entry z_{t,i,j} (Sec. IV-B: "z is a Rademacher
  * vector").  One Philox block covers 128 consecutive indices j of one worker row:
  * counter = (j >> 7, worker, round, domain 0), key = (seed low, seed high).
- * Element j takes bit (j & 31) of output word (j >> 5) & 3.  0 -> +1, 1 -> -1. */
+ * Element j takes bit (j & 31) of output word (j >> 5) & 3.  0 -> +1, 1 -> -1.
+ * With several Hutchinson samples per step, sample s = 0, 1, ... uses the counter
+ * word 256 s in place of the domain 0 (sample 0 is the single-sample stream). */
+static inline uint32_t orc_zbit_s(uint64_t seed, uint32_t t, uint32_t i, uint32_t sample, uint64_t j)
+{
+    uint32_t ctr[4] = { (uint32_t)(j >> 7), i, t, ORC_DOMAIN_Z + 256u * sample };
+    uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    uint32_t r[4];
+    orc_philox4x32_10(ctr, key, r);
+    return (r[(j >> 5) & 3] >> (j & 31)) & 1u;
+}
+
 static inline uint32_t orc_zbit(uint64_t seed, uint32_t t, uint32_t i, uint64_t j)
 {
     uint32_t ctr[4] = { (uint32_t)(j >> 7), i, t, ORC_DOMAIN_Z };
@@ -103,17 +114,33 @@ void orc_sample_z(uint64_t seed, uint32_t t, int K, uint64_t P, float *z, uint64
 
 /* Sign bits of one whole worker row, one Philox call per 128 indices (the same
  * values as orc_zbit; only the repeated calls are saved). sgn[j] in {0,1}. */
-static void orc_zbits_row(uint64_t seed, uint32_t t, uint32_t i, uint64_t P, uint8_t *sgn)
+static void orc_zbits_row_s(uint64_t seed, uint32_t t, uint32_t i, uint32_t sample, uint64_t P,
+                            uint8_t *sgn)
 {
     uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
     for (uint64_t base = 0; base < P; base += 128) {
-        uint32_t ctr[4] = { (uint32_t)(base >> 7), i, t, ORC_DOMAIN_Z };
+        uint32_t ctr[4] = { (uint32_t)(base >> 7), i, t, ORC_DOMAIN_Z + 256u * sample };
         uint32_t r[4];
         orc_philox4x32_10(ctr, key, r);
         uint64_t end = base + 128 < P ? base + 128 : P;
         for (uint64_t j = base; j < end; ++j)
             sgn[j] = (uint8_t)((r[(j >> 5) & 3] >> (j & 31)) & 1u);
     }
+}
+
+static void orc_zbits_row(uint64_t seed, uint32_t t, uint32_t i, uint64_t P, uint8_t *sgn)
+{
+    orc_zbits_row_s(seed, t, i, 0u, P, sgn);
+}
+
+/* z of Hutchinson sample `sample`, per element from the definition. */
+void orc_sample_z_s(uint64_t seed, uint32_t t, uint32_t sample, int K, uint64_t P, float *z,
+                    uint64_t ld)
+{
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < K; ++i)
+        for (uint64_t j = 0; j < P; ++j)
+            z[(uint64_t)i * ld + j] = orc_zbit_s(seed, t, (uint32_t)i, sample, j) ? -1.0f : 1.0f;
 }
 
 /* z bits as bytes [K][P] (for bit-exact comparison with the device generator). */
@@ -167,11 +194,15 @@ void orc_hutchinson_row(const float *hvp, const uint8_t *sgn, uint64_t P, float 
 /* ------------------------------------------------------------------------- */
 #include <stdlib.h>
 
-int orc_local_step(float *x, float *m, float *v, uint32_t *step,
-                   const float *grad, const float *hvp, int K, uint64_t P, uint64_t ld,
-                   const orc_segment *segs, int nseg, uint64_t z_seed, uint32_t t,
-                   float lr, float beta1, float beta2, float eps, float hessian_power,
-                   float weight_decay, const uint8_t *active)
+/* n_samples Hutchinson samples per step (Sec. IV-B: diag(H) ~ (1/n) sum_s z_s (.) H z_s):
+ * hvp holds sample s at hvp + s * sample_stride, each [K][ld]; the products are summed
+ * in ascending s and divided by n once (n = 1: no division), then averaged spatially. */
+int orc_local_step_n(float *x, float *m, float *v, uint32_t *step,
+                     const float *grad, const float *hvp, int n_samples, uint64_t sample_stride,
+                     int K, uint64_t P, uint64_t ld,
+                     const orc_segment *segs, int nseg, uint64_t z_seed, uint32_t t,
+                     float lr, float beta1, float beta2, float eps, float hessian_power,
+                     float weight_decay, const uint8_t *active)
 {
     int err = 0;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -203,6 +234,17 @@ int orc_local_step(float *x, float *m, float *v, uint32_t *step,
 
         orc_zbits_row(z_seed, t, (uint32_t)i, P, sgn);
         orc_hutchinson_row(hvp + (uint64_t)i * ld, sgn, P, d);
+        if (n_samples > 1) {
+            for (int sidx = 1; sidx < n_samples; ++sidx) {
+                const float *hs = hvp + (uint64_t)sidx * sample_stride + (uint64_t)i * ld;
+                orc_zbits_row_s(z_seed, t, (uint32_t)i, (uint32_t)sidx, P, sgn);
+                orc_hutchinson_row(hs, sgn, P, dbar);            /* dbar as scratch */
+                for (uint64_t j = 0; j < P; ++j)
+                    d[j] = (float)((real)d[j] + (real)dbar[j]);
+            }
+            for (uint64_t j = 0; j < P; ++j)
+                d[j] = (float)((real)d[j] / (real)n_samples);
+        }
         orc_spatial_average(d, P, segs, nseg, dbar);
 
         for (uint64_t j = 0; j < P; ++j) {
@@ -232,6 +274,16 @@ int orc_local_step(float *x, float *m, float *v, uint32_t *step,
         free(sgn); free(d); free(dbar);
     }
     return err;
+}
+
+int orc_local_step(float *x, float *m, float *v, uint32_t *step,
+                   const float *grad, const float *hvp, int K, uint64_t P, uint64_t ld,
+                   const orc_segment *segs, int nseg, uint64_t z_seed, uint32_t t,
+                   float lr, float beta1, float beta2, float eps, float hessian_power,
+                   float weight_decay, const uint8_t *active)
+{
+    return orc_local_step_n(x, m, v, step, grad, hvp, 1, 0, K, P, ld, segs, nseg, z_seed, t, lr,
+                            beta1, beta2, eps, hessian_power, weight_decay, active);
 }
 
 /* ------------------------------------------------------------------------- */
