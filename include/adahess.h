@@ -53,6 +53,7 @@ extern "C" {
 #define AH_MAX_WORKERS  256        /* K <= 256                                              */
 #define AH_MAX_BLOCK    128        /* spatial block kh*kw <= 128 (covers 11 x 11 kernels)   */
 #define AH_MAX_HIST     32         /* history depth p of the raw score <= 32                */
+#define AH_MAX_SAMPLES  8          /* Hutchinson samples per step <= 8                      */
 #define AH_ROUND_AUTO   0xFFFFFFFFu
 #define AH_STATIC_SCRATCH_ENTRIES (1 << 17)  /* doubles per row of the built-in scratch     */
 #define AH_DEVICE_NONE  (-2)       /* ah_alloc.device: bookkeeping-only handle, no GPU      */
@@ -86,6 +87,9 @@ typedef struct {
                              skips this step entirely (its x, m, v, step count stay)        */
     int want_dist;        /* 1 = also compute n2_i = ||x_i - c||^2 after the step, for all
                              K workers, into the handle (read by dw_weights_next)           */
+    int n_samples;        /* Hutchinson samples per step, 1 .. AH_MAX_SAMPLES; 0 means 1     */
+    uint64_t hvp_sample_stride; /* elements from sample s to sample s + 1 inside hvp (a
+                             multiple of 4, at least K * ld); ignored for one sample        */
 } ah_hyper;
 
 /* Hyper-parameters of one first-order local step (sgd_local_step). */
@@ -174,9 +178,17 @@ int ah_broadcast_center(ah_ctx *h);
  * z internally (no z buffer is read there). */
 int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t ld);
 
+/* The same for Hutchinson sample `sample` (0 .. AH_MAX_SAMPLES-1) when a step uses
+ * several: sample s replaces the last counter word 0 by 256 s.  Sample 0 is
+ * ah_sample_z. */
+int ah_sample_z_n(ah_ctx *h, uint64_t z_seed, uint32_t round, uint32_t sample, float *dst,
+                  uint64_t ld);
+
 /* One local AdaHessian step of every active worker (Sec. IV-B; Eq. 4), fused in
  * one pass over the state.  For worker i with t_i = its step count after this step:
- *     D      = z (.) hvp                     Hutchinson estimate, one sample
+ *     D      = z (.) hvp                     Hutchinson estimate; with n_samples = n > 1
+ *                                            D = (sum_s z_s (.) hvp_s) / n, summed in
+ *                                            ascending s, hvp_s = hvp + s * stride
  *     Dbar   = block mean of D               spatial averaging inside each tensor,
  *                                            summed in ascending index order
  *     m      = beta1*m + (1-beta1)*grad

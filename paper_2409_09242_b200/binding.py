@@ -26,14 +26,14 @@ AH_OK = 0
 AH_ERR_INVALID_ARG, AH_ERR_ALIGN, AH_ERR_SEGMENTS, AH_ERR_ALLOC = -1, -2, -3, -4
 AH_ERR_CUDA, AH_ERR_STATE, AH_ERR_INTERNAL, AH_ERR_TOO_LARGE = -5, -6, -7, -8
 AH_STATIC_SCRATCH_ENTRIES = 1 << 17
-AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST = 256, 128, 32
+AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST, AH_MAX_SAMPLES = 256, 128, 32, 8
 AH_ROUND_AUTO = 0xFFFFFFFF
 AH_DEVICE_NONE = -2
 (AH_X, AH_M, AH_V, AH_CENTER, AH_NORM2, AH_STEP, AH_UHIST, AH_DOWN_UNTIL, AH_ROUND,
  AH_INFO, AH_RUNS, AH_TILES) = range(12)
 
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
-           "ah_broadcast_center", "ah_sample_z", "ah_local_step", "dw_config",
+           "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
            "dw_order_next", "easgd_exchange_async", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
@@ -47,7 +47,8 @@ class ah_segment(C.Structure):
 class ah_hyper(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
                 ("eps", C.c_float), ("hessian_power", C.c_float), ("weight_decay", C.c_float),
-                ("round", C.c_uint32), ("active", C.POINTER(C.c_uint8)), ("want_dist", C.c_int)]
+                ("round", C.c_uint32), ("active", C.POINTER(C.c_uint8)), ("want_dist", C.c_int),
+                ("n_samples", C.c_int), ("hvp_sample_stride", C.c_uint64)]
 
 
 class sgd_hyper(C.Structure):
@@ -69,6 +70,7 @@ _lib.ah_state_set.argtypes = [_vp, C.c_int, C.c_int, _vp, C.c_int]
 _lib.ah_state_get.argtypes = [_vp, C.c_int, C.c_int, _vp, C.c_int]
 _lib.ah_broadcast_center.argtypes = [_vp]
 _lib.ah_sample_z.argtypes = [_vp, C.c_uint64, C.c_uint32, _vp, C.c_uint64]
+_lib.ah_sample_z_n.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_uint32, _vp, C.c_uint64]
 _lib.ah_local_step.argtypes = [_vp, _vp, _vp, C.c_uint64, C.c_uint64, C.POINTER(ah_hyper)]
 _lib.dw_config.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), C.c_double]
 _lib.dw_weights_next.argtypes = [_vp, C.c_float, C.POINTER(C.c_float)]
@@ -282,10 +284,21 @@ class Handle:
                                      dst.stride(0)), "ah_sample_z")
         return dst
 
+    def ah_sample_z_n(self, z_seed, round_, sample, dst):
+        self._check(_lib.ah_sample_z_n(self._h, int(z_seed), int(round_), int(sample),
+                                       _dev_ptr(dst, "dst"), dst.stride(0)), "ah_sample_z_n")
+        return dst
+
     def ah_local_step(self, grad, hvp, z_seed, lr, beta1=0.9, beta2=0.999, eps=1e-4,
                       hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
                       want_dist=False):
-        if grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
+        """hvp: [K, ld] for one Hutchinson sample, or [n, K, ld] for n samples per step."""
+        n_samples, sample_stride = 1, 0
+        if hvp.dim() == 3:
+            n_samples, sample_stride = hvp.shape[0], hvp.stride(0)
+            if hvp.stride(2) != 1 or hvp.shape[1:] != grad.shape or hvp.stride(1) != grad.stride(0):
+                raise ValueError("hvp: [n, K, ld] with the shape and row stride of grad")
+        elif grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
             raise ValueError("grad and hvp must share shape and row stride")
         act = None
         if active is not None:
@@ -294,9 +307,9 @@ class Handle:
                 raise ValueError("active: K bytes")
         hy = ah_hyper(lr, beta1, beta2, eps, hessian_power, weight_decay, int(round_),
                       act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None,
-                      1 if want_dist else 0)
+                      1 if want_dist else 0, int(n_samples), int(sample_stride))
         self._check(_lib.ah_local_step(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
-                                       grad.stride(0), int(z_seed), C.byref(hy)), "ah_local_step")
+                                       grad.stride(-2), int(z_seed), C.byref(hy)), "ah_local_step")
 
     def sgd_local_step(self, grad, lr, momentum=0.0, active=None, want_dist=False):
         act = None

@@ -277,14 +277,20 @@ int ah_broadcast_center(ah_ctx *h)
     return AH_OK;
 }
 
-int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t ld)
+int ah_sample_z_n(ah_ctx *h, uint64_t z_seed, uint32_t round, uint32_t sample, float *dst,
+                  uint64_t ld)
 {
-    if (!h || !dst || ld < h->P) return AH_ERR_INVALID_ARG;
+    if (!h || !dst || ld < h->P || sample >= AH_MAX_SAMPLES) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
     AH_CUDA(h, launch_sample_z(dst, ld, h->P, h->K, (uint32_t)(z_seed & 0xffffffffu),
-                               (uint32_t)(z_seed >> 32), round, h->stream));
+                               (uint32_t)(z_seed >> 32), round, sample, h->stream));
     h->launches += 1;
     return AH_OK;
+}
+
+int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t ld)
+{
+    return ah_sample_z_n(h, z_seed, round, 0u, dst, ld);
 }
 
 int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
@@ -297,8 +303,17 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0 || ((uintptr_t)hvp & 15u) != 0)
         return AH_ERR_ALIGN;
 
+    const int nsamp = hy->n_samples > 0 ? hy->n_samples : 1;
+    if (nsamp > AH_MAX_SAMPLES) return AH_ERR_INVALID_ARG;
+    if (nsamp > 1) {
+        if (hy->hvp_sample_stride < (uint64_t)(h->K - 1) * ld + h->P) return AH_ERR_INVALID_ARG;
+        if ((hy->hvp_sample_stride & 3u) != 0) return AH_ERR_ALIGN;
+    }
+
     const bool dist = hy->want_dist != 0;
     StepParams p;
+    p.nsamp = (uint32_t)nsamp;
+    p.sample_stride = nsamp > 1 ? hy->hvp_sample_stride : 0;
     p.x = h->x; p.m = h->m; p.v = h->v; p.c = h->c;
     p.grad = grad; p.hvp = hvp;
     p.partials = h->partials;

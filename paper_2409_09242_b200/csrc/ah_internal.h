@@ -92,6 +92,8 @@ struct StepParams {
     uint32_t ntiles_pad;       // power of two >= ntiles
     uint32_t key0, key1, round;
     float lr, beta1, beta2, omb1, omb2, eps, hpow, wd;
+    uint32_t nsamp;            // Hutchinson samples per step (1 .. AH_MAX_SAMPLES)
+    uint64_t sample_stride;    // elements between consecutive samples in hvp
     uint32_t nrows;            // worker rows to process (all K when distances are wanted)
     uint32_t nitems;           // nrows * ntiles
     WorkerConst w[AH_MAX_WORKERS];
@@ -116,7 +118,7 @@ cudaError_t launch_norm2_finalize(double *partials, double *scratch, uint32_t nt
                                   uint32_t ntiles_pad, int K, double *norm2, cudaStream_t s);
 cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s);
 cudaError_t launch_sample_z(float *dst, uint64_t ld, uint32_t P, int K, uint32_t key0,
-                            uint32_t key1, uint32_t round, cudaStream_t s);
+                            uint32_t key1, uint32_t round, uint32_t sample, cudaStream_t s);
 cudaError_t launch_broadcast(float *x, const float *c, uint64_t lds, int K, cudaStream_t s);
 
 // Philox4x32-10 (Salmon et al., SC'11), usable on both sides.

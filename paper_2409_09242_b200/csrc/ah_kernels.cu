@@ -246,6 +246,13 @@ struct __align__(128) Stage {
     float hv[kTile + 2 * kHalo];           // element j lives at hv[j - t0 + kHalo]
 };
 
+// With n > 1 Hutchinson samples per step, samples 1 .. n-1 of every stage live behind
+// the fixed part of shared memory: their Philox words and their Hessian-vector tile.
+struct __align__(128) ExtraSample {
+    uint32_t zw[kStageGroups][4];
+    float hv[kTile + 2 * kHalo];
+};
+
 template <bool DIST>
 struct __align__(128) Shared {
     Stage<DIST> stage[kStages];
@@ -281,12 +288,37 @@ __device__ __forceinline__ void block_means_any(float *base, uint32_t nblk, uint
     }
 }
 
-template <int POWMODE, bool WD, bool DIST>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+// Hutchinson estimate of four consecutive elements (Sec. IV-B): z (.) hvp for one
+// sample; with MULTI the sum over the samples in ascending order, divided by their
+// number.  hidx indexes the stage's hvp arrays, gidx its Philox groups, j is the
+// element's index in the row (it selects the word and the bit of the signs).
+template <bool MULTI, bool DIST>
+__device__ __forceinline__ float4 hutchinson4(const Stage<DIST> &st, const ExtraSample *xs,
+                                              uint32_t nsamp, uint32_t hidx, uint32_t gidx,
+                                              uint32_t j, float fn, float rn)
+{
+    const uint32_t wsel = (j >> 5) & 3u, shift = j & 31u;
+    float4 D = apply_signs(ld_vec(&st.hv[hidx]), (st.zw[gidx][wsel] >> shift) & 0xFu);
+    if constexpr (MULTI) {
+        for (uint32_t q = 0; q + 1u < nsamp; ++q) {
+            const float4 e = apply_signs(ld_vec(&xs[q].hv[hidx]), (xs[q].zw[gidx][wsel] >> shift) & 0xFu);
+            D.x = __fadd_rn(D.x, e.x); D.y = __fadd_rn(D.y, e.y);
+            D.z = __fadd_rn(D.z, e.z); D.w = __fadd_rn(D.w, e.w);
+        }
+        D.x = div_by_const(D.x, fn, rn); D.y = div_by_const(D.y, fn, rn);
+        D.z = div_by_const(D.z, fn, rn); D.w = div_by_const(D.w, fn, rn);
+    }
+    return D;
+}
+
+template <int POWMODE, bool WD, bool DIST, bool MULTI>
+__global__ void __launch_bounds__(kThreads, MULTI ? 3 : kCtasPerSm)
 local_step_kernel(const __grid_constant__ StepParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Shared<DIST> &sh = *reinterpret_cast<Shared<DIST> *>(smem_raw);
+    ExtraSample *extra = reinterpret_cast<ExtraSample *>(smem_raw + sizeof(Shared<DIST>));
+    const uint32_t nextra = MULTI ? p.nsamp - 1u : 0u;     // extra samples per stage
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
@@ -336,8 +368,13 @@ local_step_kernel(const __grid_constant__ StepParams p)
             if (act) {
                 const uint32_t g0 = ea0 >> 7;
                 const uint32_t ng = ((ea1 - 1u) >> 7) - g0 + 1u;
-                if ((uint32_t)lane < ng)
+                if ((uint32_t)lane < ng) {
                     philox4x32_10(g0 + lane, i, p.round, kDomainZ, p.key0, p.key1, st.zw[lane]);
+                    if constexpr (MULTI)
+                        for (uint32_t q = 0; q < nextra; ++q)
+                            philox4x32_10(g0 + lane, i, p.round, kDomainZ + 256u * (q + 1u), p.key0,
+                                          p.key1, extra[s * nextra + q].zw[lane]);
+                }
             }
             if (lane == 0) {
                 st.worker = i; st.t0 = t0; st.nvalid = nvalid;
@@ -351,8 +388,15 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 const uint64_t so = (uint64_t)i * p.lds + t0;
                 uint64_t *bar = &sh.full[s];
                 if (act) {
-                    mbar_arrive_expect_tx(bar, 4u * row_bytes + hv_bytes + (DIST ? row_bytes : 0u));
+                    mbar_arrive_expect_tx(bar, 4u * row_bytes + (1u + nextra) * hv_bytes +
+                                                   (DIST ? row_bytes : 0u));
                     bulk_load(&st.hv[ea0 + kHalo - t0], p.hvp + (uint64_t)i * p.ld + ea0, hv_bytes, bar);
+                    if constexpr (MULTI)
+                        for (uint32_t q = 0; q < nextra; ++q)
+                            bulk_load(&extra[s * nextra + q].hv[ea0 + kHalo - t0],
+                                      p.hvp + (uint64_t)(q + 1u) * p.sample_stride +
+                                          (uint64_t)i * p.ld + ea0,
+                                      hv_bytes, bar);
                     bulk_load(st.g, p.grad + (uint64_t)i * p.ld + t0, row_bytes, bar);
                     bulk_load(st.x, p.x + so, row_bytes, bar);
                     bulk_load(st.m, p.m + so, row_bytes, bar);
@@ -386,6 +430,8 @@ local_step_kernel(const __grid_constant__ StepParams p)
         Stage<DIST> &st = sh.stage[s];
         const uint32_t i = st.worker, t0 = st.t0, nvalid = st.nvalid, flags = st.flags;
         if (flags & kItemEnd) break;
+        const ExtraSample *xs = extra + s * nextra;
+        const float fn = (float)p.nsamp, rn = __frcp_rn(fn);
         float4 xn[kPasses];
 
         if (!(flags & kItemDistanceOnly)) {
@@ -394,10 +440,9 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 // ---- z (.) hvp in place over the widened range
                 const uint32_t ea0 = st.ea0, ea1 = (st.e1 + 3u) & ~3u, g0 = ea0 >> 7;
                 for (uint32_t q = ctid; q < (ea1 - ea0) >> 2; q += kConsumers) {
-                    const uint32_t j = ea0 + 4u * q;
-                    const uint32_t word = st.zw[(j >> 7) - g0][(j >> 5) & 3u];
-                    float *ptr = &st.hv[j + kHalo - t0];
-                    st_vec(ptr, apply_signs(ld_vec(ptr), (word >> (j & 31u)) & 0xFu));
+                    const uint32_t j = ea0 + 4u * q, hidx = j + kHalo - t0;
+                    st_vec(&st.hv[hidx],
+                           hutchinson4<MULTI, DIST>(st, xs, p.nsamp, hidx, (j >> 7) - g0, j, fn, rn));
                 }
                 consumer_sync();
                 // ---- block means in place, one thread per block
@@ -424,11 +469,9 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
                 if (off < nvalid) {
                     const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
-                    float4 D = ld_vec(&st.hv[off + kHalo]);
-                    if (!(flags & kItemAverage)) {
-                        const uint32_t word = st.zw[off >> 7][(off >> 5) & 3u];
-                        D = apply_signs(D, (word >> (off & 31u)) & 0xFu);
-                    }
+                    const float4 D = (flags & kItemAverage)
+                        ? ld_vec(&st.hv[off + kHalo])
+                        : hutchinson4<MULTI, DIST>(st, xs, p.nsamp, off + kHalo, off >> 7, off, fn, rn);
                     const float4 g = ld_vec(&st.g[off]);
                     float4 x = ld_vec(&st.x[off]), m = ld_vec(&st.m[off]), v = ld_vec(&st.v[off]);
                     if (nv == 4) {
@@ -562,14 +605,15 @@ exchange_kernel(const __grid_constant__ ExchangeParams p)
 
 // Rademacher vectors as +-1.0f (one thread per four consecutive elements).
 __global__ void __launch_bounds__(256)
-sample_z_kernel(float *dst, uint64_t ld, uint32_t P, uint32_t key0, uint32_t key1, uint32_t round)
+sample_z_kernel(float *dst, uint64_t ld, uint32_t P, uint32_t key0, uint32_t key1, uint32_t round,
+                uint32_t sample)
 {
     const uint32_t q = blockIdx.x * 256u + threadIdx.x;
     const uint32_t j = 4u * q;
     const int i = blockIdx.y;
     if (q >= (P + 3u) / 4u) return;
     uint32_t w[4];
-    philox4x32_10(j >> 7, (uint32_t)i, round, kDomainZ, key0, key1, w);
+    philox4x32_10(j >> 7, (uint32_t)i, round, kDomainZ + 256u * sample, key0, key1, w);
     const uint32_t word = w[(j >> 5) & 3u];
     float *row = dst + (uint64_t)i * ld;
     for (uint32_t e = 0; e < 4u && j + e < P; ++e)
@@ -588,15 +632,19 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-template <int POWMODE, bool WD, bool DIST>
+template <int POWMODE, bool WD, bool DIST, bool MULTI>
 static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream_t s)
 {
-    auto kernel = local_step_kernel<POWMODE, WD, DIST>;
-    const size_t smem = sizeof(Shared<DIST>);
+    auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI>;
+    const size_t smem = sizeof(Shared<DIST>) +
+                        (MULTI ? (size_t)kStages * (p.nsamp - 1u) * sizeof(ExtraSample) : 0);
     static bool configured = false;      // per instantiation
+    static int ctas_for_nsamp[AH_MAX_SAMPLES + 1] = {};
     if (!configured) {
+        const size_t most = sizeof(Shared<DIST>) +
+                            (MULTI ? (size_t)kStages * (AH_MAX_SAMPLES - 1) * sizeof(ExtraSample) : 0);
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+                                             (int)most);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
@@ -604,7 +652,18 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
         configured = true;
     }
     if (p.nitems == 0) return cudaSuccess;
-    const uint32_t resident = (uint32_t)sm_count * (uint32_t)kCtasPerSm;
+    int ctas = kCtasPerSm;
+    if (MULTI) {                         // the extra samples decide how many CTAs fit
+        if (ctas_for_nsamp[p.nsamp] == 0) {
+            int fit = 0;
+            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, kThreads, smem);
+            if (e != cudaSuccess) return e;
+            if (fit < 1) return cudaErrorInvalidConfiguration;
+            ctas_for_nsamp[p.nsamp] = fit;
+        }
+        ctas = ctas_for_nsamp[p.nsamp];
+    }
+    const uint32_t resident = (uint32_t)sm_count * (uint32_t)ctas;
     const uint32_t grid = p.nitems < resident ? p.nitems : resident;
     kernel<<<grid, kThreads, smem, s>>>(p);
     return cudaGetLastError();
@@ -613,8 +672,11 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
 template <int POWMODE, bool WD>
 static cudaError_t launch_step_dist(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
 {
-    return want_dist ? launch_step_one<POWMODE, WD, true>(p, sm_count, s)
-                     : launch_step_one<POWMODE, WD, false>(p, sm_count, s);
+    if (p.nsamp > 1u)
+        return want_dist ? launch_step_one<POWMODE, WD, true, true>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, true>(p, sm_count, s);
+    return want_dist ? launch_step_one<POWMODE, WD, true, false>(p, sm_count, s)
+                     : launch_step_one<POWMODE, WD, false, false>(p, sm_count, s);
 }
 
 cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
@@ -648,11 +710,11 @@ cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s)
 }
 
 cudaError_t launch_sample_z(float *dst, uint64_t ld, uint32_t P, int K, uint32_t key0,
-                            uint32_t key1, uint32_t round, cudaStream_t s)
+                            uint32_t key1, uint32_t round, uint32_t sample, cudaStream_t s)
 {
     const unsigned nvec = (P + 3u) / 4u;
     const dim3 grid((nvec + 255u) / 256u, (unsigned)K);
-    sample_z_kernel<<<grid, 256, 0, s>>>(dst, ld, P, key0, key1, round);
+    sample_z_kernel<<<grid, 256, 0, s>>>(dst, ld, P, key0, key1, round, sample);
     return cudaGetLastError();
 }
 

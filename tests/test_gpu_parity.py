@@ -172,6 +172,63 @@ def test_exchange_alpha_zero_is_identity(B, torch):
     h.close()
 
 
+# ------------------------------------------- several Hutchinson samples per step
+@pytest.mark.parametrize("sample", [0, 1, 7])
+def test_sample_z_n_bit_exact(B, torch, sample):
+    K, P = 3, 184_837
+    h = B.Handle(K, P, [])
+    dst = torch.empty(K, W.padded_ld(P), device="cuda")
+    h.ah_sample_z_n(0xFEEDFACE12345678, 9, sample, dst)
+    want = oracle.load("omp").sample_z_s(0xFEEDFACE12345678, 9, sample, K, P)
+    assert np.array_equal(dst[:, :P].cpu().numpy(), want)
+    h.close()
+
+
+@pytest.mark.parametrize("n", [2, 3, 4, 8])
+@pytest.mark.parametrize("layout", ["odd", "resnet18"])
+def test_local_step_n_samples_matches_oracle(B, torch, n, layout):
+    if layout == "odd":
+        segs, P = ODD_SEGS, ODD_P
+    else:
+        lay = W.resnet18_layout(16)
+        segs, P = W.segments(lay), W.total_params(lay)
+    K, ld = 3, W.padded_ld(P)
+    rng = np.random.default_rng(n * 100 + P)
+    theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
+    h = B.Handle(K, P, segs)
+    ref = OracleState(theta0, K, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    for t in range(1, 6):
+        g = np.zeros((K, ld), np.float32)
+        hv = np.zeros((n, K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        hv[:, :, :P] = rng.standard_normal((n, K, P)).astype(np.float32) * np.float32(0.1)
+        active = None if t != 3 else np.array([1, 0, 1], np.uint8)
+        dist = t % 2 == 0
+        h.ah_local_step(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda(), Z_SEED, lr=0.01,
+                        round_=t, active=active, want_dist=dist)
+        ref.local_step(g, hv, Z_SEED, t, lr=0.01, active=active, want_dist=dist)
+        if dist:
+            assert np.array_equal(h.ah_state_get(B.AH_NORM2), ref.norm2), t
+    for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v)):
+        assert np.array_equal(h.ah_state_get(which), want), which
+    h.close()
+
+
+def test_n_samples_argument_checks(B, torch):
+    K, P = 2, 1000
+    h = B.Handle(K, P, [])
+    g = torch.zeros(K, P, device="cuda")
+    with pytest.raises(B.AdaHessError) as e:
+        h.ah_local_step(g, torch.zeros(B.AH_MAX_SAMPLES + 1, K, P, device="cuda"), 1, lr=0.1)
+    assert e.value.status == B.AH_ERR_INVALID_ARG
+    hy = B.ah_hyper(0.1, 0.9, 0.999, 1e-4, 1.0, 0.0, 1, None, 0, 2, P)     # samples would overlap
+    hv = torch.zeros(2, K, P, device="cuda")
+    assert B.raw().ah_local_step(h._h, g.data_ptr(), hv.data_ptr(), P, 1, C.byref(hy)) == B.AH_ERR_INVALID_ARG
+    h.close()
+
+
 # --------------------------------------------------- asynchronous exchange
 @pytest.mark.parametrize("K,P", [(1, 7), (3, 1000), (4, 4099), (7, 2048), (16, 10_001), (64, 3001),
                                  (256, 1030)])
