@@ -161,7 +161,7 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
                              active=mask if frozen else None)
         else:
             h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
-                            **HYPER)
+                            **HYPER)      # hv is [K, ld], or [n, K, ld] with --samples n
         n_act = int(mask.sum()) if frozen else K
         worker_steps += n_act
         if events is not None:
@@ -206,9 +206,14 @@ def gpu_arm(args):
     dev = torch.device("cuda", local_rank)
 
     # synthetic inputs, resident in HBM before the timed region
-    pair_bytes = 2 * K * ld * 4
+    pair_bytes = (1 + args.samples) * K * ld * 4
     n_pool = max(1, min(args.pool, int(24e9 // pair_bytes)))
     pool = [W.gaussian_pair_torch(layout, K, DATA_SEED + 1 + 1000 * r + rank, dev) for r in range(n_pool)]
+    if args.samples > 1:         # n Hutchinson samples per step: hvp becomes [n, K, ld]
+        pool = [(g, torch.stack([hv] + [W.gaussian_pair_torch(layout, K, DATA_SEED + 7 + 1000 * r + 50 * q
+                                                              + rank, dev)[1]
+                                        for q in range(1, args.samples)]))
+                for r, (g, hv) in enumerate(pool)]
     h = binding.Handle(K, P, segs)
     h.ah_state_set(binding.AH_CENTER, W.theta0_torch(layout, DATA_SEED + rank, dev))
     h.ah_broadcast_center()
@@ -256,30 +261,30 @@ def gpu_arm(args):
     withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex]
     # algorithmic bytes of a launch: 32 per update; a distance round also reads the
     # master row once and the x of every worker that sat the step out
-    bpu = {"adahessian": 32, "sgd": 12, "msgd": 20}[args.method]
+    bpu = {"adahessian": 28 + 4 * args.samples, "sgd": 12, "msgd": 20}[args.method]
     if args.method != "adahessian":
         dom, dom_name = plain + withd, "sgd_step"       # no distance rounds with a fixed alpha
         dom_bytes = sum(bpu * P * n for _, n in dom) / len(dom)
     elif plain:
         dom, dom_name = plain, "local_step"
-        dom_bytes = sum(32 * P * n for _, n in dom) / len(dom)
+        dom_bytes = sum(bpu * P * n for _, n in dom) / len(dom)
     else:
         dom, dom_name = withd, "local_step+dist"
-        dom_bytes = sum(32 * P * n + 4 * P * (K - n) + 4 * P for _, n in dom) / len(dom)
+        dom_bytes = sum(bpu * P * n + 4 * P * (K - n) + 4 * P for _, n in dom) / len(dom)
     dom_ms = sum(d for d, _ in dom) / len(dom)
     peak, peak_kind = measured_hbm_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
     if (args.method == "adahessian" and NCU_TRAFFIC["sources_sha256"] == kernel_sources_hash()
             and NCU_TRAFFIC["dram_bytes_per_update"]):
-        traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0
+        traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0 if args.samples == 1 else None
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": traffic,
                 "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
                 "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
-    run_bytes = bpu * P * worker_steps + 8 * P * exchanged + (12 if bpu == 32 else 8) * P * args.steps
+    run_bytes = bpu * P * worker_steps + 8 * P * exchanged + (12 if args.method == "adahessian" else 8) * P * args.steps
     whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
     # the exchange kernel alone: 8 bytes per (arriving worker, parameter) + 8 per parameter
@@ -318,8 +323,8 @@ def gpu_arm(args):
             ems = float(tmax.item())
         e2e = {"value": round(e2e_ws * P * world / (ems * 1e-3) / 1e9, 3),
                "unit": "G param-updates/s", "steps": e2e_steps,
-               "h2d_bytes_per_step": (pair_bytes if bpu == 32 else pair_bytes // 2) * tau,
-               "d2h_bytes_per_step": 8 * K if bpu == 32 else 0}
+               "h2d_bytes_per_step": (pair_bytes if args.method == "adahessian" else K * ld * 4) * tau,
+               "d2h_bytes_per_step": 8 * K if args.method == "adahessian" else 0}
 
     out = {
         "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
@@ -334,6 +339,7 @@ def gpu_arm(args):
                    "local_step": {"adahessian": "AdaHessian, dynamic weights",
                                   "sgd": "SGD, fixed alpha (EASGD)",
                                   "msgd": "SGD with momentum 0.5, fixed alpha (EAMSGD)"}[args.method],
+                   "hutchinson_samples": args.samples,
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
                    "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
@@ -382,6 +388,10 @@ def oracle_periods(args, layout, periods, warm):
     import oracle
     segs, P = W.segments(layout), W.total_params(layout)
     pool = W.gaussian_pool_np(layout, K, 2, DATA_SEED + 1)
+    if args.samples > 1:
+        more = [W.gaussian_pool_np(layout, K, 2, DATA_SEED + 7 + 50 * q) for q in range(1, args.samples)]
+        pool = [(g, np.ascontiguousarray(np.stack([hv] + [m[r][1] for m in more])))
+                for r, (g, hv) in enumerate(pool)]
     st = oracle.OracleState(W.theta0_np(layout, DATA_SEED), K, segs, variant="omp")
     alpha = alpha_for(K)
     t, t_start, worker_steps = 0, None, 0
@@ -457,6 +467,7 @@ def main():
                     help="all workers against the same master value, or one at a time")
     ap.add_argument("--method", default="adahessian", choices=["adahessian", "sgd", "msgd"],
                     help="local step: the paper's method, or the EASGD / EAMSGD comparison methods")
+    ap.add_argument("--samples", type=int, default=1, help="Hutchinson samples per step (paper: 1)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
