@@ -53,13 +53,13 @@ HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weigh
 # DRAM bytes per parameter update of the fused local-step kernel, from one ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch / (K * P)), and the hash
 # of the kernel sources it was taken on.  Reported only while the sources are unchanged.
-NCU_TRAFFIC = {"sources_sha256": "1cca58c8068d2b49fe52e249e8e5b7055ba94e780a9c2b2bba29f2f657b99434",
-               "dram_bytes_per_update": 1.446244e9 / 46_758_048}
+NCU_TRAFFIC = {"sources_sha256": "5e76b9a43fd00c9859378f931ad5bb80d788e1c4c5f8058e131a4b1d5da6447d",
+               "dram_bytes_per_update": 1.443466e9 / 46_758_048}
 
 
 def kernel_sources_hash() -> str:
     h = hashlib.sha256()
-    for fn in ("ah_kernels.cu", "ah_internal.h"):
+    for fn in ("ah_kernels.cu", "ah_internal.h", "ah_device.cuh"):
         with open(os.path.join(ROOT, "paper_2409_09242_b200", "csrc", fn), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
@@ -128,6 +128,21 @@ class ClockSampler:
                     reasons.add(n)
         return {"sm_mhz": statistics.median(clocks) if clocks else None, "sm_max_mhz": mx,
                 "samples": len(clocks), "reasons": sorted(reasons)}
+
+
+def max_over_ranks(ms, dist, device):
+    """The slowest rank's time: what a multi-GPU number is quoted on."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_updates_per_second(updates_per_rank, world, ms):
+    """G parameter updates per second over all replicas (every rank does the same work)."""
+    return updates_per_rank * world / (ms * 1e-3) / 1e9
 
 
 def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
@@ -247,13 +262,9 @@ def gpu_arm(args):
     ms = start.elapsed_time(stop)
     clocks = sampler.stop() if rank == 0 else None
     launches = h.ah_launch_count() - launches0
-    if dist is not None:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(ms, dist, dev)
     # parameter updates actually performed: a frozen straggler takes no step
-    updates = worker_steps * P * world
-    value = updates / (ms * 1e-3) / 1e9
+    value = whole_job_updates_per_second(worker_steps * P, world, ms)
 
     # per-launch duration of the fused local-step kernel (plain rounds; the rounds that
     # also measure distances are listed beside it)
@@ -317,11 +328,8 @@ def gpu_arm(args):
         stop.record()
         barrier()
         ems = start.elapsed_time(stop)
-        if dist is not None:
-            tmax = torch.tensor([ems], device=dev)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            ems = float(tmax.item())
-        e2e = {"value": round(e2e_ws * P * world / (ems * 1e-3) / 1e9, 3),
+        ems = max_over_ranks(ems, dist, dev)
+        e2e = {"value": round(whole_job_updates_per_second(e2e_ws * P, world, ems), 3),
                "unit": "G param-updates/s", "steps": e2e_steps,
                "h2d_bytes_per_step": (pair_bytes if args.method == "adahessian" else K * ld * 4) * tau,
                "d2h_bytes_per_step": 8 * K if args.method == "adahessian" else 0}
