@@ -104,6 +104,8 @@ class Oracle:
         L.orc_sample_z_s.restype = None
         L.orc_norm2.argtypes = [pf, pf, C.c_int, C.c_uint64, pd]
         L.orc_norm2.restype = None
+        L.orc_ln.argtypes = [C.c_double]
+        L.orc_ln.restype = C.c_double
         L.orc_u_from_norm2.argtypes = [C.c_double]
         L.orc_u_from_norm2.restype = C.c_double
         for f in (L.orc_h1, L.orc_h2):
@@ -166,6 +168,12 @@ class Oracle:
         n2 = np.empty(K, np.float64)
         self.lib.orc_norm2(_f32(x), _f32(c), K, P, n2.ctypes.data_as(C.POINTER(C.c_double)))
         return n2
+
+    def ln(self, x):
+        return self.lib.orc_ln(float(x))
+
+    def u_from_norm2(self, n2):
+        return self.lib.orc_u_from_norm2(float(n2))
 
     def h1(self, a, alpha, kappa):
         return self.lib.orc_h1(a, alpha, kappa)
