@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "ah_ctx.h"
+#include "ah_ln.cuh"
 
 using namespace ah;
 
@@ -462,7 +463,7 @@ int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *we
     for (int i = 0; i < h->K; ++i) {
         double *ring = &h->uhist[(size_t)i * depth];
         const double n2 = h->norm2_last[i];
-        const double u = 0.5 * log(n2 > 1e-300 ? n2 : 1e-300);   // log of the 2-norm
+        const double u = u_from_norm2(n2);                       // log of the 2-norm
         if (h->ring_filled) memmove(ring + 1, ring, (size_t)h->p_hist * sizeof(double));
         else for (int j = 1; j < depth; ++j) ring[j] = u;
         ring[0] = u;
