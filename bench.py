@@ -146,7 +146,7 @@ def whole_job_updates_per_second(updates_per_rank, world, ms):
 
 
 def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
-               method="adahessian"):
+               method="adahessian", sync_free=False):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
     memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
@@ -183,12 +183,16 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
             e1.record()
             events.append((e0, e1, ex, n_act))
         if ex:
-            w = None if first_order else h.dw_weights_next(alpha)
+            on_device = sync_free and not first_order      # weights computed on the device
+            w = None if (first_order or on_device) else h.dw_weights_next(alpha)
             if ex_events is not None:
                 x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 x0.record()
-            if asynchronous:
-                h.easgd_exchange_async(mask, w, alpha, h.dw_order_next(ORDER_SEED, t))
+            order = h.dw_order_next(ORDER_SEED, t) if asynchronous else None
+            if on_device:
+                h.easgd_exchange_dynamic(mask, alpha, order, asynchronous)
+            elif asynchronous:
+                h.easgd_exchange_async(mask, w, alpha, order)
             else:
                 h.easgd_exchange(mask, w, alpha)
             if ex_events is not None:
@@ -242,7 +246,7 @@ def gpu_arm(args):
     t = 0
     asyn = args.exchange == "async"
     for _ in range(args.warmup):
-        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method)
+        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -254,7 +258,7 @@ def gpu_arm(args):
     worker_steps = exchanged = 0
     for _ in range(args.steps):
         t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events,
-                                method=args.method)
+                                method=args.method, sync_free=args.sync_free)
         worker_steps += ws
         exchanged += exd
     stop.record()
@@ -317,7 +321,7 @@ def gpu_arm(args):
         sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
         t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn,
-                             method=args.method)
+                             method=args.method)      # the end-to-end leg reads the weights back
         barrier()
         start.record()
         e2e_ws = 0
@@ -348,6 +352,7 @@ def gpu_arm(args):
                                   "sgd": "SGD, fixed alpha (EASGD)",
                                   "msgd": "SGD with momentum 0.5, fixed alpha (EAMSGD)"}[args.method],
                    "hutchinson_samples": args.samples,
+                   "weights": "on the device, no host wait" if args.sync_free else "on the host, one wait per period",
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
                    "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
@@ -475,6 +480,8 @@ def main():
                     help="all workers against the same master value, or one at a time")
     ap.add_argument("--method", default="adahessian", choices=["adahessian", "sgd", "msgd"],
                     help="local step: the paper's method, or the EASGD / EAMSGD comparison methods")
+    ap.add_argument("--sync-free", action="store_true",
+                    help="dynamic weights computed on the device: no host wait in a period")
     ap.add_argument("--samples", type=int, default=1, help="Hutchinson samples per step (paper: 1)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -131,9 +131,11 @@ enum {
     AH_INFO = 9,       /* uint32 [4]   {tiles, runs, elements per tile, row stride} (get only)  */
     AH_RUNS = 10,      /* uint32 [runs][4]  {start, end, block, reciprocal}: the row cut into
                           maximal runs of equal spatial block (get only, host)              */
-    AH_TILES = 11      /* uint32 [tiles][4] {first run, e0, e1, flags}: each tile's range
+    AH_TILES = 11,     /* uint32 [tiles][4] {first run, e0, e1, flags}: each tile's range
                           widened to whole spatial blocks [e0, e1); flags bit 0 = the tile
                           touches a block > 1 (get only, host)                              */
+    AH_WEIGHTS = 12    /* float  [2K]  h2[0..K) then h1[0..K) of the last
+                          easgd_exchange_dynamic (get only, host)                           */
 };
 
 /* ---- life cycle ------------------------------------------------------------ */
@@ -255,6 +257,19 @@ int dw_mask_next(ah_ctx *h, uint64_t seed, uint32_t round, double p_fail, int ma
  * weights: host pointer, 2K floats as written by dw_weights_next, or NULL
  * (h1_i = h2_i = alpha for all i).  alpha is ignored when weights != NULL. */
 int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha);
+
+/* The exchange of one round with the dynamic weights computed on the device: the same
+ * rule as dw_weights_next (Sec. V-B, Eqs. 10-11, h1/h2), same history ring, same bits,
+ * fed by the distances of the last want_dist step, followed by the weighted exchange
+ * (Eqs. 12-13) of easgd_exchange (asynchronous == 0; order ignored) or
+ * easgd_exchange_async (asynchronous != 0; order as there, NULL = ascending).  Nothing
+ * is copied to the host and the call does not wait, so a whole communication period
+ * can be queued ahead of the GPU.  The coefficients used can be read afterwards with
+ * ah_state_get(AH_WEIGHTS); the history with AH_UHIST.  Host and device forms of the
+ * rule may be mixed freely on one handle.
+ * Errors: STATE when no distances are pending, INVALID_ARG for a bad order, CUDA. */
+int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, float alpha,
+                           const uint16_t *order, int asynchronous);
 
 /* ---- data overlap -------------------------------------------------------------- */
 

@@ -30,12 +30,12 @@ AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST, AH_MAX_SAMPLES = 256, 128, 32, 8
 AH_ROUND_AUTO = 0xFFFFFFFF
 AH_DEVICE_NONE = -2
 (AH_X, AH_M, AH_V, AH_CENTER, AH_NORM2, AH_STEP, AH_UHIST, AH_DOWN_UNTIL, AH_ROUND,
- AH_INFO, AH_RUNS, AH_TILES) = range(12)
+ AH_INFO, AH_RUNS, AH_TILES, AH_WEIGHTS) = range(13)
 
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -84,6 +84,8 @@ _lib.dw_partition.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, C.
 _lib.dw_order_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.POINTER(C.c_uint16)]
 _lib.easgd_exchange_async.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
                                       C.POINTER(C.c_uint16)]
+_lib.easgd_exchange_dynamic.argtypes = [_vp, C.POINTER(C.c_uint8), C.c_float, C.POINTER(C.c_uint16),
+                                        C.c_int]
 _lib.ah_distances_static.argtypes = [_vp, C.c_uint64, _vp, C.c_int, C.c_uint64, _vp, _vp]
 _lib.ah_status_string.argtypes = [C.c_int]
 _lib.ah_status_string.restype = C.c_char_p
@@ -257,6 +259,8 @@ class Handle:
             a = np.empty(shape, np.float32)
         elif which == AH_CENTER:
             a = np.empty(self.P, np.float32)
+        elif which == AH_WEIGHTS:
+            a = np.empty(2 * self.K, np.float32)
         elif which == AH_NORM2:
             a = np.empty(self.K, np.float64)
         elif which == AH_UHIST:
@@ -384,6 +388,19 @@ class Handle:
                 raise ValueError("order: K entries")
             o = order.ctypes.data_as(C.POINTER(C.c_uint16))
         self._check(_lib.easgd_exchange_async(self._h, m, w, alpha, o), "easgd_exchange_async")
+
+    def easgd_exchange_dynamic(self, worker_mask=None, alpha=0.0, order=None, asynchronous=False):
+        m = o = None
+        if worker_mask is not None:
+            worker_mask = np.ascontiguousarray(worker_mask, np.uint8)
+            m = worker_mask.ctypes.data_as(C.POINTER(C.c_uint8))
+        if order is not None:
+            order = np.ascontiguousarray(order, np.uint16)
+            if order.size != self.K:
+                raise ValueError("order: K entries")
+            o = order.ctypes.data_as(C.POINTER(C.c_uint16))
+        self._check(_lib.easgd_exchange_dynamic(self._h, m, alpha, o, 1 if asynchronous else 0),
+                    "easgd_exchange_dynamic")
 
     def ah_launch_count(self):
         return int(_lib.ah_launch_count(self._h))

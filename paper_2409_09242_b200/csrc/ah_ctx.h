@@ -27,6 +27,9 @@ struct ah_ctx {
     double *partials = nullptr, *scratch = nullptr;
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
+    uint32_t *ring_flag_dev = nullptr;   // device copy of ring_filled
+    double *uhist_dev = nullptr;   // device copy of the history ring, [K][p_hist + 1]
+    float *weights_dev = nullptr;  // [2K] coefficients of the last dynamic exchange
     ah::Run *runs = nullptr;
     ah::TileInfo *tiles = nullptr;
     uint32_t nruns = 0;
@@ -34,7 +37,9 @@ struct ah_ctx {
     // host state
     double *norm2_host = nullptr;  // pinned copy of norm2_dev (status word + K doubles)
     cudaEvent_t norm2_ready = nullptr;
-    bool norm2_pending = false;    // a want_dist step has been enqueued since the last read
+    bool norm2_pending = false;    // distances of a want_dist step not yet used by a weight rule
+    bool norm2_unread = false;     // ... and not yet copied into norm2_last
+    int ring_home = 0;             // 0: the host copy of the ring is current, 1: the device copy
     double norm2_last[AH_MAX_WORKERS];
     uint32_t step[AH_MAX_WORKERS];
     uint32_t down_until[AH_MAX_WORKERS];
@@ -58,4 +63,9 @@ inline int ah_cuda_fail(ah_ctx *h, cudaError_t e)
 
 namespace ah {
 int finish_distances(ah_ctx *h);   // ah_host.cu
+int ring_to_host(ah_ctx *h);
+int ring_to_device(ah_ctx *h);
+int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
+                  const uint16_t *order, const float *weights_dev, ExchangeParams &p);
+cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu
 }

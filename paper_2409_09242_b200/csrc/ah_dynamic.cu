@@ -1,0 +1,56 @@
+// Exchange rounds without a host round trip: the dynamic weights of Sec. V-B are
+// computed on the device from the distances the preceding local step left there, and
+// the exchange kernel reads them from device memory.  The host never waits, so the
+// next period's launches can be queued while this one still runs.
+#include "ah_ctx.h"
+#include "ah_weights.cuh"
+
+namespace ah {
+
+// One thread per worker: the weighting rule for worker i (the same function the host
+// entry points run), on the device copy of the history ring.
+__global__ void __launch_bounds__(AH_MAX_WORKERS)
+dynamic_weights_kernel(const __grid_constant__ WeightRule rule, const double *norm2, double *uhist,
+                       uint32_t *ring_flag, float *weights, int nworkers)
+{
+    const int i = threadIdx.x;
+    const bool filled = *ring_flag != 0u;
+    __syncthreads();                               // everybody has read the flag
+    if (i < nworkers)
+        weight_rule_step(rule, norm2[i], uhist + (size_t)i * (rule.p_hist + 1), filled, &weights[i],
+                         &weights[nworkers + i]);
+    if (i == 0) *ring_flag = 1u;
+}
+
+}  // namespace ah
+
+using namespace ah;
+
+extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, float alpha,
+                                      const uint16_t *order, int asynchronous)
+{
+    if (!h) return AH_ERR_INVALID_ARG;
+    if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
+    ExchangeParams p;
+    int rc = fill_exchange(h, worker_mask, nullptr, alpha, asynchronous ? order : nullptr,
+                           h->weights_dev, p);
+    if (rc != AH_OK) return rc;
+    if ((rc = ring_to_device(h)) != AH_OK) return rc;
+
+    WeightRule rule;
+    rule.p_hist = h->p_hist;
+    for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < h->p_hist ? h->coef[j] : 0.0;
+    rule.kappa = h->kappa;
+    rule.alpha = (double)alpha;
+    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1, h->uhist_dev,
+                                                                 h->ring_flag_dev, h->weights_dev, h->K);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->launches += 1;
+    h->norm2_pending = false;                      // these distances have fed the rule
+    if (p.nact == 0) return AH_OK;                 // the history advances even if nobody arrives
+    e = asynchronous ? launch_exchange_in_order(p, h->stream) : launch_exchange(p, h->stream);
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->launches += 1;
+    return AH_OK;
+}

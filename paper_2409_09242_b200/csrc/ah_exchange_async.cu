@@ -49,7 +49,7 @@ exchange_async_kernel(const __grid_constant__ ExchangeParams p)
             xv[u] = ldg4(p.x + (uint64_t)p.idx[a + u] * p.lds + col);
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const float h1 = p.h1[a + u], h2 = p.h2[a + u];
+            const float h1 = exchange_h1(p, a + u), h2 = exchange_h2(p, a + u);
             meet(xv[u].x, c.x, h1, h2);
             meet(xv[u].y, c.y, h1, h2);
             meet(xv[u].z, c.z, h1, h2);
@@ -59,7 +59,7 @@ exchange_async_kernel(const __grid_constant__ ExchangeParams p)
     }
     for (; a < p.nact; ++a) {
         float4 xv = ldg4(p.x + (uint64_t)p.idx[a] * p.lds + col);
-        const float h1 = p.h1[a], h2 = p.h2[a];
+        const float h1 = exchange_h1(p, a), h2 = exchange_h2(p, a);
         meet(xv.x, c.x, h1, h2);
         meet(xv.y, c.y, h1, h2);
         meet(xv.z, c.z, h1, h2);
@@ -109,6 +109,24 @@ int easgd_exchange_async(ah_ctx *h, const uint8_t *worker_mask, const float *wei
 {
     if (!h) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
+    ExchangeParams p;
+    const int rc = ah::fill_exchange(h, worker_mask, weights, alpha, order, nullptr, p);
+    if (rc != AH_OK) return rc;
+    if (p.nact == 0) return AH_OK;                // nobody arrives: nothing moves
+    const cudaError_t e = launch_exchange_async(p, h->stream);
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->launches += 1;
+    return AH_OK;
+}
+
+}  // extern "C"
+
+// Arrival list and coefficients of one exchange: the workers that take part, in
+// `order` (null: ascending), with coefficients from `weights` (host, 2K floats), from
+// `weights_dev` (device, same layout) or all equal to alpha.
+int ah::fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
+                      const uint16_t *order, const float *weights_dev, ExchangeParams &p)
+{
     if (order) {                                  // must name every worker exactly once
         bool seen[AH_MAX_WORKERS] = {};
         for (int q = 0; q < h->K; ++q) {
@@ -116,9 +134,10 @@ int easgd_exchange_async(ah_ctx *h, const uint8_t *worker_mask, const float *wei
             seen[order[q]] = true;
         }
     }
-    ExchangeParams p;
     p.x = h->x; p.c = h->c; p.lds = h->lds;
     p.nvec = (uint32_t)(h->lds / 4);
+    p.wdev = weights_dev;
+    p.nworkers = h->K;
     p.nact = 0;
     for (int q = 0; q < h->K; ++q) {
         const int i = order ? (int)order[q] : q;
@@ -128,11 +147,10 @@ int easgd_exchange_async(ah_ctx *h, const uint8_t *worker_mask, const float *wei
         p.h1[p.nact] = weights ? weights[h->K + i] : alpha;
         p.nact += 1;
     }
-    if (p.nact == 0) return AH_OK;                // nobody arrives: nothing moves
-    const cudaError_t e = launch_exchange_async(p, h->stream);
-    if (e != cudaSuccess) return ah_cuda_fail(h, e);
-    h->launches += 1;
     return AH_OK;
 }
 
-}  // extern "C"
+cudaError_t ah::launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s)
+{
+    return launch_exchange_async(p, s);
+}

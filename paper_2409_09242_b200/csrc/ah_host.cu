@@ -9,7 +9,7 @@
 #include <vector>
 
 #include "ah_ctx.h"
-#include "ah_ln.cuh"
+#include "ah_weights.cuh"
 
 using namespace ah;
 
@@ -37,7 +37,7 @@ int cuda_fail(ah_ctx *h, cudaError_t e)
     } while (0)
 
 struct Layout {
-    size_t x, m, v, c, partials, scratch, norm2, sched, runs, tiles, total;
+    size_t x, m, v, c, partials, scratch, norm2, sched, uhist, weights, runs, tiles, total;
 };
 
 // Offsets of every array inside the workspace (each 256-byte aligned).
@@ -56,7 +56,9 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.partials = take((size_t)K * ntp * sizeof(double));
     L.scratch = take((size_t)K * ntp * sizeof(double));
     L.norm2 = take((size_t)(AH_MAX_WORKERS + 1) * sizeof(double));
-    L.sched = take(2 * sizeof(uint32_t));
+    L.sched = take(4 * sizeof(uint32_t));                 // item counter, exit counter, ring flag
+    L.uhist = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
+    L.weights = take(2 * (size_t)K * sizeof(float));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
     L.total = off;
@@ -131,6 +133,36 @@ void reset_history(ah_ctx *h)
 
 }  // namespace
 
+// The history ring of the weighting rule has a host copy and a device copy; ring_home
+// says which one is current.  These bring the other side up to date.
+int ah::ring_to_host(ah_ctx *h)
+{
+    if (!h->has_device || h->ring_home == 0) return AH_OK;
+    AH_CUDA(h, cudaStreamSynchronize(h->stream));
+    const size_t depth = (size_t)h->p_hist + 1;
+    AH_CUDA(h, cudaMemcpy(h->uhist.data(), h->uhist_dev, (size_t)h->K * depth * sizeof(double),
+                          cudaMemcpyDeviceToHost));
+    uint32_t filled = 0;
+    AH_CUDA(h, cudaMemcpy(&filled, h->ring_flag_dev, sizeof(filled), cudaMemcpyDeviceToHost));
+    h->ring_filled = (int)filled;
+    h->ring_home = 0;
+    return AH_OK;
+}
+
+int ah::ring_to_device(ah_ctx *h)
+{
+    if (h->ring_home == 1) return AH_OK;
+    const size_t depth = (size_t)h->p_hist + 1;
+    const uint32_t filled = (uint32_t)h->ring_filled;
+    // pageable sources: the calls return once the data has been staged
+    AH_CUDA(h, cudaMemcpyAsync(h->uhist_dev, h->uhist.data(), (size_t)h->K * depth * sizeof(double),
+                               cudaMemcpyHostToDevice, h->stream));
+    AH_CUDA(h, cudaMemcpyAsync(h->ring_flag_dev, &filled, sizeof(filled), cudaMemcpyHostToDevice,
+                               h->stream));
+    h->ring_home = 1;
+    return AH_OK;
+}
+
 // After a step has left the tile partials of ||x_i - c||^2 in the workspace: finish
 // the pairwise tree on the device and start the copy of the K doubles (and the status
 // word in front of them) to pinned host memory.
@@ -143,6 +175,7 @@ int ah::finish_distances(ah_ctx *h)
                                cudaMemcpyDeviceToHost, h->stream));
     AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
     h->norm2_pending = true;
+    h->norm2_unread = true;
     return AH_OK;
 }
 
@@ -227,6 +260,9 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->scratch = (double *)(base + L.scratch);
     h->norm2_dev = (double *)(base + L.norm2);
     h->sched = (uint32_t *)(base + L.sched);
+    h->ring_flag_dev = h->sched + 2;
+    h->uhist_dev = (double *)(base + L.uhist);
+    h->weights_dev = (float *)(base + L.weights);
     h->runs = (Run *)(base + L.runs);
     h->tiles = (TileInfo *)(base + L.tiles);
 
@@ -377,6 +413,17 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
         return AH_OK;
     }
     if (on_device) return AH_ERR_INVALID_ARG;
+    if (which == AH_WEIGHTS) {                 // coefficients of the last dynamic exchange
+        if (!to_user || !h->has_device) return to_user ? AH_ERR_STATE : AH_ERR_INVALID_ARG;
+        AH_CUDA(h, cudaMemcpyAsync(user, h->weights_dev, 2 * (size_t)h->K * sizeof(float),
+                                   cudaMemcpyDeviceToHost, h->stream));
+        AH_CUDA(h, cudaStreamSynchronize(h->stream));
+        return AH_OK;
+    }
+    if (which == AH_UHIST || which == AH_ROUND) {
+        const int rc = ring_to_host(h);
+        if (rc != AH_OK) return rc;
+    }
     void *ptr;
     size_t bytes;
     uint32_t round_info[2];
@@ -402,9 +449,10 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
     default: return AH_ERR_INVALID_ARG;
     }
     if (to_user) {
-        if (which == AH_NORM2 && h->norm2_pending) {
+        if (which == AH_NORM2 && h->norm2_unread) {
             AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
             memcpy(h->norm2_last, h->norm2_host + 1, h->K * sizeof(double));
+            h->norm2_unread = false;
         }
         memcpy(user, ptr, bytes);
     } else {
@@ -413,7 +461,8 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
             h->calls = round_info[0];
             h->ring_filled = (int)round_info[1];
         }
-        if (which == AH_NORM2) h->norm2_pending = false;
+        if (which == AH_NORM2) { h->norm2_pending = false; h->norm2_unread = false; }
+        if (which == AH_UHIST || which == AH_ROUND) h->ring_home = 0;    // the host copy leads again
     }
     return AH_OK;
 }
@@ -425,7 +474,14 @@ int ah_state_set(ah_ctx *h, int which, int worker, const void *src, int src_on_d
 
 int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device)
 {
-    if (h && h->has_device) AH_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (h && h->has_device) {
+        // the device status word is looked at whenever the host waits for the stream anyway
+        uint32_t status = 0;
+        AH_CUDA(h, cudaMemcpyAsync(&status, h->norm2_dev, sizeof(status), cudaMemcpyDeviceToHost,
+                                   h->stream));
+        AH_CUDA(h, cudaStreamSynchronize(h->stream));
+        if (status != 0u) return AH_ERR_INTERNAL;
+    }
     return state_copy(h, which, worker, dst, dst_on_device, true);
 }
 
@@ -437,6 +493,7 @@ int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
     for (int j = 0; j < p_hist; ++j) h->coef[j] = c[j];
     h->kappa = kappa;
     reset_history(h);
+    h->ring_home = 0;
     return AH_OK;
 }
 
@@ -446,6 +503,7 @@ int dw_weights_next(ah_ctx *h, float alpha, float *weights)
     if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
     AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
     h->norm2_pending = false;
+    h->norm2_unread = false;
     if (*reinterpret_cast<const uint32_t *>(h->norm2_host) != 0u) return AH_ERR_INTERNAL;
     return dw_weights_from_norm2(h, h->norm2_host + 1, alpha, weights);
 }
@@ -453,30 +511,19 @@ int dw_weights_next(ah_ctx *h, float alpha, float *weights)
 int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *weights)
 {
     if (!h || !norm2 || !weights) return AH_ERR_INVALID_ARG;
+    const int rc = ring_to_host(h);
+    if (rc != AH_OK) return rc;
     memcpy(h->norm2_last, norm2, h->K * sizeof(double));
 
+    WeightRule rule;
+    rule.p_hist = h->p_hist;
+    memcpy(rule.coef, h->coef, sizeof(rule.coef));
+    rule.kappa = h->kappa;
+    rule.alpha = (double)alpha;
     const int depth = h->p_hist + 1;
-    const double a_rate = (double)alpha, kap = h->kappa;
-    const double slope_worker = (1.0 - a_rate) / kap;    // h1 falls from 1 to alpha on [kappa, 0]
-    const double slope_master = -a_rate / kap;           // h2 rises from 0 to alpha on [kappa, 0]
-    float *to_master = weights, *to_worker = weights + h->K;
-    for (int i = 0; i < h->K; ++i) {
-        double *ring = &h->uhist[(size_t)i * depth];
-        const double n2 = h->norm2_last[i];
-        const double u = u_from_norm2(n2);                       // log of the 2-norm
-        if (h->ring_filled) memmove(ring + 1, ring, (size_t)h->p_hist * sizeof(double));
-        else for (int j = 1; j < depth; ++j) ring[j] = u;
-        ring[0] = u;
-        double score = 0.0;                               // Eqs. 10-11
-        for (int j = 0; j < h->p_hist; ++j) score = score + h->coef[j] * (ring[j] - ring[j + 1]);
-        double w_worker, w_master;
-        if (score < kap)        { w_worker = 1.0; w_master = 0.0; }
-        else if (score <= 0.0)  { w_worker = 1.0 + slope_worker * (score - kap);
-                                  w_master = slope_master * score + a_rate; }
-        else                    { w_worker = a_rate; w_master = a_rate; }
-        to_worker[i] = (float)w_worker;
-        to_master[i] = (float)w_master;
-    }
+    for (int i = 0; i < h->K; ++i)
+        weight_rule_step(rule, h->norm2_last[i], &h->uhist[(size_t)i * depth], h->ring_filled != 0,
+                         &weights[i], &weights[h->K + i]);
     h->ring_filled = 1;
     return AH_OK;
 }
@@ -516,16 +563,8 @@ int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, 
     if (!h) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
     ExchangeParams p;
-    p.x = h->x; p.c = h->c; p.lds = h->lds;
-    p.nvec = (uint32_t)(h->lds / 4);
-    p.nact = 0;
-    for (int i = 0; i < h->K; ++i) {
-        if (worker_mask && !worker_mask[i]) continue;
-        p.idx[p.nact] = (uint16_t)i;
-        p.h2[p.nact] = weights ? weights[i] : alpha;
-        p.h1[p.nact] = weights ? weights[h->K + i] : alpha;
-        p.nact += 1;
-    }
+    const int rc = fill_exchange(h, worker_mask, weights, alpha, nullptr, nullptr, p);
+    if (rc != AH_OK) return rc;
     if (p.nact == 0) return AH_OK;     // nobody reaches the master: nothing moves
     AH_CUDA(h, launch_exchange(p, h->stream));
     h->launches += 1;

@@ -110,7 +110,24 @@ struct ExchangeParams {
     uint16_t idx[AH_MAX_WORKERS];   // their indices, ascending
     float h1[AH_MAX_WORKERS];       // compacted to the same order
     float h2[AH_MAX_WORKERS];
+    const float *wdev;              // not null: coefficients come from device memory instead,
+                                    // h2 of worker i at wdev[i], h1 at wdev[nworkers + i]
+    int nworkers;
 };
+
+#ifdef __CUDACC__
+// Coefficients of the a-th arriving worker, from the launch parameters or, when the
+// weights were computed on the device, from memory.
+__device__ __forceinline__ float exchange_h1(const ExchangeParams &p, int a)
+{
+    return p.wdev ? p.wdev[p.nworkers + p.idx[a]] : p.h1[a];
+}
+
+__device__ __forceinline__ float exchange_h2(const ExchangeParams &p, int a)
+{
+    return p.wdev ? p.wdev[p.idx[a]] : p.h2[a];
+}
+#endif
 
 // Kernel launchers (ah_kernels.cu).  Each returns the cudaError_t of the launch.
 cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);

@@ -588,13 +588,13 @@ exchange_kernel(const __grid_constant__ ExchangeParams p)
             xv[u] = ld_vec(p.x + (uint64_t)p.idx[a + u] * p.lds + col);
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            pull4(xv[u], acc, c, p.h1[a + u], p.h2[a + u]);
+            pull4(xv[u], acc, c, exchange_h1(p, a + u), exchange_h2(p, a + u));
             st_vec(p.x + (uint64_t)p.idx[a + u] * p.lds + col, xv[u]);
         }
     }
     for (; a < p.nact; ++a) {
         float4 xv = ld_vec(p.x + (uint64_t)p.idx[a] * p.lds + col);
-        pull4(xv, acc, c, p.h1[a], p.h2[a]);
+        pull4(xv, acc, c, exchange_h1(p, a), exchange_h2(p, a));
         st_vec(p.x + (uint64_t)p.idx[a] * p.lds + col, xv);
     }
     float4 cn;

@@ -28,6 +28,8 @@ class RunConfig:
     alpha: float | None = None      # None: min(0.05, 0.8 / K)
     dynamic: bool = True            # dynamic weights (else fixed alpha)
     asynchronous: bool = False      # workers reach the master one at a time, seeded order
+    sync_free: str = "no"           # "yes": weights on the device (easgd_exchange_dynamic);
+                                    # "mixed": device and host forms of the rule alternate
     method: str = "adahessian"      # local step: "adahessian", "sgd" or "msgd" (momentum)
     momentum: float = 0.5
     scripted: list = field(default_factory=list)
@@ -85,20 +87,31 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         if ex:
             log["exchanges"] += 1
             w = h2 = h1 = None
-            if cfg.dynamic:
-                w = h.dw_weights_next(alpha)
-                h2, h1 = ref.weights_next(alpha)
-                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
-                log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], h2) and
-                                             np.array_equal(w[cfg.K:], h1))
+            on_device = cfg.dynamic and (cfg.sync_free == "yes" or
+                                         (cfg.sync_free == "mixed" and log["exchanges"] % 2 == 1))
+            order_g = order_o = None
             if cfg.asynchronous:
                 order_g = h.dw_order_next(ORDER_SEED, t)
                 order_o = ref.order_next(ORDER_SEED, t)
                 log["orders_equal"] &= bool(np.array_equal(order_g, order_o))
-                h.easgd_exchange_async(mask_g, w, alpha, order_g)
+            if cfg.dynamic:
+                h2, h1 = ref.weights_next(alpha)
+            if on_device:
+                h.easgd_exchange_dynamic(mask_g, alpha, order_g, cfg.asynchronous)
+                w = h.ah_state_get(binding.AH_WEIGHTS)
+            elif cfg.dynamic:
+                w = h.dw_weights_next(alpha)
+            if cfg.dynamic:
+                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+                log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], h2) and
+                                             np.array_equal(w[cfg.K:], h1))
+            if cfg.asynchronous:
+                if not on_device:
+                    h.easgd_exchange_async(mask_g, w, alpha, order_g)
                 ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
             else:
-                h.easgd_exchange(mask_g, w, alpha)
+                if not on_device:
+                    h.easgd_exchange(mask_g, w, alpha)
                 ref.exchange(mask_o, h2, h1, alpha=alpha)
         if check_every and t % check_every == 0:
             assert tolerance_violations(h.ah_state_get(binding.AH_X), ref.x) == 0, t

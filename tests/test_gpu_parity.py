@@ -286,6 +286,54 @@ def test_async_rounds_resnet18_shape_reduced(B, torch):
     h.close()
 
 
+# --------------------------------------- weights on the device, no host round trip
+@pytest.mark.parametrize("asyn,mode", [(False, "yes"), (True, "yes"), (False, "mixed"), (True, "mixed")])
+def test_dynamic_exchange_on_device_matches_oracle(B, torch, asyn, mode):
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=120, tau=2,
+                    p_fail=0.3, alpha=0.1 if asyn else None, asynchronous=asyn, sync_free=mode)
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"] and log["orders_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert log["exchanges"] == 60
+    h.close()
+
+
+def test_dynamic_exchange_custom_rule_and_errors(B, torch):
+    # a deeper history with other coefficients and threshold; K = 256 fills the weight kernel
+    K, P, p_hist = 256, 1500, 7
+    rng = np.random.default_rng(60)
+    c = rng.dirichlet(np.ones(p_hist))
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    h = B.Handle(K, P, [])
+    h.dw_config(p_hist, c, -0.25)
+    ref = OracleState(theta0, K, [], p_hist=p_hist, c=c, kappa=-0.25)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    with pytest.raises(B.AdaHessError) as e:
+        h.easgd_exchange_dynamic(None, 0.003)              # no distances yet
+    assert e.value.status == B.AH_ERR_STATE
+    zeros = torch.zeros(K, W.padded_ld(P), device="cuda")
+    for t in range(1, 13):
+        x = (theta0[None] + rng.standard_normal((K, P)).astype(np.float32) *
+             rng.uniform(0.01, 1.0, (K, 1)).astype(np.float32))
+        h.ah_state_set(B.AH_X, x)
+        ref.x[:] = x
+        h.ah_local_step(zeros, zeros, 1, lr=0.0, active=np.zeros(K, np.uint8), want_dist=True)
+        ref.norm2 = oracle.load("omp").norm2(ref.x, ref.center)
+        h.easgd_exchange_dynamic(None, 0.003)
+        h2, h1 = ref.weights_next(0.003)
+        ref.exchange(None, h2, h1)
+        w = h.ah_state_get(B.AH_WEIGHTS)
+        assert np.array_equal(w[:K], h2) and np.array_equal(w[K:], h1), t
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST, p_hist=p_hist), ref.uhist)
+    assert np.array_equal(h.ah_state_get(B.AH_X), ref.x)
+    assert np.array_equal(h.ah_state_get(B.AH_CENTER), ref.center)
+    h.close()
+
+
 # ------------------------------------------- first-order local steps (EASGD / EAMSGD)
 @pytest.mark.parametrize("K,P", [(1, 1), (2, 1023), (3, 4097), (4, 184_837), (8, 4 * 1024 * 5), (5, 8193)])
 @pytest.mark.parametrize("delta", [0.0, 0.5])
