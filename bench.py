@@ -146,7 +146,7 @@ def whole_job_updates_per_second(updates_per_rank, world, ms):
 
 
 def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
-               method="adahessian", sync_free=False):
+               method="adahessian", sync_free=False, fused=False):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
     memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
@@ -174,6 +174,12 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         if first_order:
             h.sgd_local_step(g, SGD_LR, SGD_MOMENTUM if method == "msgd" else 0.0,
                              active=mask if frozen else None)
+        elif fused and ex:
+            # the whole exchange round in one pass; the rule's coefficients lag one period
+            h.ah_local_step_exchange(g, hv, Z_SEED, round_=t, active=mask if frozen else None,
+                                     want_dist=True, worker_mask=mask, alpha=alpha,
+                                     order=h.dw_order_next(ORDER_SEED, t) if asynchronous else None,
+                                     asynchronous=asynchronous, lagged=True, **HYPER)
         else:
             h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
                             **HYPER)      # hv is [K, ld], or [n, K, ld] with --samples n
@@ -182,7 +188,9 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         if events is not None:
             e1.record()
             events.append((e0, e1, ex, n_act))
-        if ex:
+        if ex and fused and not first_order:
+            exchanged += int(mask.sum())
+        elif ex:
             on_device = sync_free and not first_order      # weights computed on the device
             w = None if (first_order or on_device) else h.dw_weights_next(alpha)
             if ex_events is not None:
@@ -246,7 +254,7 @@ def gpu_arm(args):
     t = 0
     asyn = args.exchange == "async"
     for _ in range(args.warmup):
-        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free)
+        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -258,7 +266,7 @@ def gpu_arm(args):
     worker_steps = exchanged = 0
     for _ in range(args.steps):
         t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events,
-                                method=args.method, sync_free=args.sync_free)
+                                method=args.method, sync_free=args.sync_free, fused=args.fused)
         worker_steps += ws
         exchanged += exd
     stop.record()
@@ -299,7 +307,12 @@ def gpu_arm(args):
                 "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
                 "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
-    run_bytes = bpu * P * worker_steps + 8 * P * exchanged + (12 if args.method == "adahessian" else 8) * P * args.steps
+    if args.fused and args.method == "adahessian":
+        # fused exchange rounds: x crosses HBM once; the master row is read and written once
+        run_bytes = bpu * P * worker_steps + 8 * P * args.steps
+    else:
+        run_bytes = (bpu * P * worker_steps + 8 * P * exchanged +
+                     (12 if args.method == "adahessian" else 8) * P * args.steps)
     whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
     # the exchange kernel alone: 8 bytes per (arriving worker, parameter) + 8 per parameter
@@ -352,6 +365,8 @@ def gpu_arm(args):
                                   "sgd": "SGD, fixed alpha (EASGD)",
                                   "msgd": "SGD with momentum 0.5, fixed alpha (EAMSGD)"}[args.method],
                    "hutchinson_samples": args.samples,
+                   "exchange_rounds": "one pass (step + pull), weights one period behind" if args.fused
+                                      else "local step, then exchange kernel",
                    "weights": "on the device, no host wait" if args.sync_free else "on the host, one wait per period",
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
                    "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
@@ -480,8 +495,11 @@ def main():
                     help="all workers against the same master value, or one at a time")
     ap.add_argument("--method", default="adahessian", choices=["adahessian", "sgd", "msgd"],
                     help="local step: the paper's method, or the EASGD / EAMSGD comparison methods")
-    ap.add_argument("--sync-free", action="store_true",
-                    help="dynamic weights computed on the device: no host wait in a period")
+    ap.add_argument("--host-weights", dest="sync_free", action="store_false",
+                    help="dynamic weights computed on the host (one wait per period) instead of "
+                         "on the device; same bits either way")
+    ap.add_argument("--fused", action="store_true",
+                    help="exchange rounds in one pass (step + pull), dynamic weights one period behind")
     ap.add_argument("--samples", type=int, default=1, help="Hutchinson samples per step (paper: 1)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -217,6 +217,29 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *hy);
 
+/* An exchange round in one pass over the state: the local step of ah_local_step
+ * followed at once, tile by tile, by the weighted pull of easgd_exchange
+ * (asynchronous == 0) or easgd_exchange_async (asynchronous != 0, order as there), so
+ * that x is read and written once instead of twice.  The result is bit for bit that of
+ * the two calls in sequence with the same coefficients:
+ *     for every column j, workers i in arrival order:
+ *         x_ij <- local step (if active_i);  n2_i += (x_ij - c_j)^2 (if hy->want_dist)
+ *         if worker_mask[i]:  pull of x_ij and the master by h1_i, h2_i   (Eqs. 12-13)
+ * The coefficients must be known before the step:
+ *   lagged == 0: weights (host, 2K floats: h2 then h1) or, when NULL, alpha for all;
+ *   lagged != 0: the dynamic rule of Sec. V-B runs on the device after this round's
+ *       distances (hy->want_dist must be 1, weights NULL) and its coefficients serve the
+ *       NEXT lagged round; the first lagged round of a handle uses alpha.  This is the
+ *       paper's "estimate of the master model": the score follows the distances with a
+ *       delay of one communication period, and no call waits for the GPU.
+ * One Hutchinson sample per step.  Memory traffic: 32 bytes per parameter update plus 8
+ * per parameter for the master row, 8 per (worker, parameter) less than the two calls.
+ * Errors: INVALID_ARG, ALIGN, STATE, CUDA. */
+int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
+                           uint64_t z_seed, const ah_hyper *hy, const uint8_t *worker_mask,
+                           const float *weights, float alpha, const uint16_t *order,
+                           int asynchronous, int lagged);
+
 /* Parameters of the dynamic weighting rule (Sec. V-B): history depth p, the
  * coefficients c_0..c_{p-1} of Eqs. 10-11 (c_0 weighs the newest difference; they
  * should sum to 1) and the threshold kappa < 0 of h1/h2.  Defaults set by ah_init:

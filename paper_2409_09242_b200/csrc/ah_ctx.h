@@ -40,6 +40,7 @@ struct ah_ctx {
     bool norm2_pending = false;    // distances of a want_dist step not yet used by a weight rule
     bool norm2_unread = false;     // ... and not yet copied into norm2_last
     int ring_home = 0;             // 0: the host copy of the ring is current, 1: the device copy
+    bool lagged_ready = false;     // weights_dev holds the rule's output of an earlier fused round
     double norm2_last[AH_MAX_WORKERS];
     uint32_t step[AH_MAX_WORKERS];
     uint32_t down_until[AH_MAX_WORKERS];
@@ -65,6 +66,7 @@ namespace ah {
 int finish_distances(ah_ctx *h);   // ah_host.cu
 int ring_to_host(ah_ctx *h);
 int ring_to_device(ah_ctx *h);
+int enqueue_weight_rule(ah_ctx *h, float alpha);   // ah_dynamic.cu
 int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                   const uint16_t *order, const float *weights_dev, ExchangeParams &p);
 cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu

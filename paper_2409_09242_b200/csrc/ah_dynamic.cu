@@ -26,6 +26,26 @@ dynamic_weights_kernel(const __grid_constant__ WeightRule rule, const double *no
 
 using namespace ah;
 
+// The weighting rule on the device, fed by the distances the last want_dist step left
+// there; its coefficients stay in weights_dev.
+int ah::enqueue_weight_rule(ah_ctx *h, float alpha)
+{
+    const int rc = ring_to_device(h);
+    if (rc != AH_OK) return rc;
+    WeightRule rule;
+    rule.p_hist = h->p_hist;
+    for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < h->p_hist ? h->coef[j] : 0.0;
+    rule.kappa = h->kappa;
+    rule.alpha = (double)alpha;
+    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1, h->uhist_dev,
+                                                                 h->ring_flag_dev, h->weights_dev, h->K);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->launches += 1;
+    h->norm2_pending = false;                      // these distances have fed the rule
+    return AH_OK;
+}
+
 extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, float alpha,
                                       const uint16_t *order, int asynchronous)
 {
@@ -35,21 +55,10 @@ extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, flo
     int rc = fill_exchange(h, worker_mask, nullptr, alpha, asynchronous ? order : nullptr,
                            h->weights_dev, p);
     if (rc != AH_OK) return rc;
-    if ((rc = ring_to_device(h)) != AH_OK) return rc;
-
-    WeightRule rule;
-    rule.p_hist = h->p_hist;
-    for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < h->p_hist ? h->coef[j] : 0.0;
-    rule.kappa = h->kappa;
-    rule.alpha = (double)alpha;
-    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1, h->uhist_dev,
-                                                                 h->ring_flag_dev, h->weights_dev, h->K);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return ah_cuda_fail(h, e);
-    h->launches += 1;
-    h->norm2_pending = false;                      // these distances have fed the rule
+    if ((rc = enqueue_weight_rule(h, alpha)) != AH_OK) return rc;
     if (p.nact == 0) return AH_OK;                 // the history advances even if nobody arrives
-    e = asynchronous ? launch_exchange_in_order(p, h->stream) : launch_exchange(p, h->stream);
+    const cudaError_t e = asynchronous ? launch_exchange_in_order(p, h->stream)
+                                       : launch_exchange(p, h->stream);
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
     h->launches += 1;
     return AH_OK;

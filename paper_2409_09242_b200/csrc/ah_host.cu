@@ -330,8 +330,21 @@ int ah_sample_z(ah_ctx *h, uint64_t z_seed, uint32_t round, float *dst, uint64_t
     return ah_sample_z_n(h, z_seed, round, 0u, dst, ld);
 }
 
-int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
-                  const ah_hyper *hy)
+namespace {
+
+// What a fused round adds to a local step: who meets the master, with which
+// coefficients, in which order.
+struct FusedExchange {
+    const uint8_t *mask;
+    const float *weights;     // host, 2K floats, or null
+    float alpha;
+    const uint16_t *order;    // host, K entries, or null (ascending)
+    bool asynchronous;
+    bool lagged;              // coefficients come from the device (previous round's rule)
+};
+
+int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
+                    const ah_hyper *hy, const FusedExchange *fx)
 {
     if (!h || !grad || !hvp || !hy || ld < h->P) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
@@ -361,18 +374,38 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
     p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
     p.key0 = (uint32_t)(z_seed & 0xffffffffu);
     p.key1 = (uint32_t)(z_seed >> 32);
-    h->calls += 1;
-    p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
     p.lr = hy->lr; p.beta1 = hy->beta1; p.beta2 = hy->beta2;
     p.omb1 = 1.0f - hy->beta1;
     p.omb2 = 1.0f - hy->beta2;
     p.eps = hy->eps; p.hpow = hy->hessian_power; p.wd = hy->weight_decay;
+    p.fused = fx ? 1u : 0u;
+    p.asynchronous = fx && fx->asynchronous ? 1u : 0u;
+    p.any_exchange = 0u;
+    p.nworkers = (uint32_t)h->K;
+    p.c_out = h->c;
+    p.wdev = fx && fx->lagged && h->lagged_ready ? h->weights_dev : nullptr;
+    if (fx && fx->order) {                        // must name every worker exactly once
+        bool seen[AH_MAX_WORKERS] = {};
+        for (int q = 0; q < h->K; ++q) {
+            if (fx->order[q] >= h->K || seen[fx->order[q]]) return AH_ERR_INVALID_ARG;
+            seen[fx->order[q]] = true;
+        }
+    }
+    h->calls += 1;
+    p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
     p.nrows = 0;
-    for (int i = 0; i < h->K; ++i) {
+    for (int q = 0; q < h->K; ++q) {
+        // a fused round walks the workers in their arrival order
+        const int i = fx && fx->asynchronous && fx->order ? (int)fx->order[q] : q;
         const bool on = !hy->active || hy->active[i] != 0;
+        const bool meets = fx && (!fx->mask || fx->mask[i] != 0);
         p.active[i] = on ? 1 : 0;
+        p.exch[i] = meets ? 1 : 0;
+        if (meets) p.any_exchange = 1u;
+        p.h2w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[i] : fx->alpha) : 0.f;
+        p.h1w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[h->K + i] : fx->alpha) : 0.f;
         if (on) h->step[i] += 1;
-        if (on || dist) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
+        if (on || dist || meets) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
         // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
         // (a worker that sat out steps has taken fewer); double, then one rounding
         const double t = (double)(h->step[i] ? h->step[i] : 1u);
@@ -382,11 +415,41 @@ int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, u
         w.rbc1 = 1.0f / w.bc1;
         w.rbc2 = 1.0f / w.bc2;
     }
-    p.nitems = p.nrows * h->ntiles;
+    p.nitems = fx ? (p.nrows ? h->ntiles : 0u) : p.nrows * h->ntiles;
     AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
     if (p.nitems) h->launches += 1;
-    if (dist) return finish_distances(h);
+    if (dist) {
+        const int rc = finish_distances(h);
+        if (rc != AH_OK) return rc;
+        if (fx && fx->lagged) {                   // the rule runs now, its output serves next time
+            const int rc2 = enqueue_weight_rule(h, fx->alpha);
+            if (rc2 != AH_OK) return rc2;
+            h->lagged_ready = true;
+        }
+    }
     return AH_OK;
+}
+
+}  // namespace
+
+int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
+                  const ah_hyper *hy)
+{
+    return local_step_impl(h, grad, hvp, ld, z_seed, hy, nullptr);
+}
+
+int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
+                           uint64_t z_seed, const ah_hyper *hy, const uint8_t *worker_mask,
+                           const float *weights, float alpha, const uint16_t *order,
+                           int asynchronous, int lagged)
+{
+    if (!hy) return AH_ERR_INVALID_ARG;
+    if (hy->n_samples > 1) return AH_ERR_INVALID_ARG;          // one Hutchinson sample when fused
+    if (lagged && (!hy->want_dist || weights)) return AH_ERR_INVALID_ARG;
+    FusedExchange fx;
+    fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;
+    fx.asynchronous = asynchronous != 0; fx.lagged = lagged != 0;
+    return local_step_impl(h, grad, hvp, ld, z_seed, hy, &fx);
 }
 
 // ---- state in / out -----------------------------------------------------------

@@ -99,6 +99,16 @@ struct StepParams {
     WorkerConst w[AH_MAX_WORKERS];
     uint16_t row[AH_MAX_WORKERS];     // row r -> worker index
     uint8_t active[AH_MAX_WORKERS];   // by worker index
+    // fused step + exchange (one pass on exchange rounds); unused otherwise
+    uint32_t fused;                   // 1: an item is a tile with all its workers, in row order
+    uint32_t asynchronous;            // 1: workers meet the master one at a time, in row order
+    uint32_t any_exchange;            // 0: nobody meets the master, it is not written
+    uint32_t nworkers;                // K, for the layout of wdev
+    float *c_out;                     // the master row, written once per tile
+    const float *wdev;                // not null: h2 of worker i at wdev[i], h1 at wdev[K + i]
+    float h1w[AH_MAX_WORKERS];        // else the coefficients by worker index
+    float h2w[AH_MAX_WORKERS];
+    uint8_t exch[AH_MAX_WORKERS];     // by worker index: meets the master this round
 };
 
 struct ExchangeParams {

@@ -233,16 +233,23 @@ __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 // p.partials[worker][tile], for every worker; a worker that sits the step out
 // contributes its unchanged x (only x and c are fetched for it).
 // ---------------------------------------------------------------------------
-enum : uint32_t { kItemAverage = 1u, kItemDistanceOnly = 2u, kItemEnd = 4u };
+enum : uint32_t {
+    kItemAverage = 1u,        // the tile touches a spatial block > 1
+    kItemDistanceOnly = 2u,   // the worker sits the step out: only x (and c) were fetched
+    kItemEnd = 4u,            // no item: the producer has left
+    kItemFirst = 8u,          // fused exchange: first worker of a tile (c was fetched with it)
+    kItemLast = 16u,          // fused exchange: last worker of a tile (the master is written back)
+    kItemExchange = 32u,      // fused exchange: this worker meets the master
+};
 
-template <bool DIST>
+template <bool HASC>
 struct __align__(128) Stage {
     uint32_t worker, t0, nvalid, flags;
     uint32_t e0, e1, run0, ea0;
     uint32_t tile, reserved[7];
     uint32_t zw[kStageGroups][4];          // Philox words of groups (ea0 >> 7) ...
     float g[kTile], x[kTile], m[kTile], v[kTile];
-    float c[DIST ? kTile : 4];
+    float c[HASC ? kTile : 4];
     float hv[kTile + 2 * kHalo];           // element j lives at hv[j - t0 + kHalo]
 };
 
@@ -253,9 +260,9 @@ struct __align__(128) ExtraSample {
     float hv[kTile + 2 * kHalo];
 };
 
-template <bool DIST>
+template <bool HASC>
 struct __align__(128) Shared {
-    Stage<DIST> stage[kStages];
+    Stage<HASC> stage[kStages];
     uint64_t full[kStages];                // producer -> consumers (bytes landed)
     uint64_t empty[kStages];               // consumers -> producer (stage drained)
     double red[2][kPasses * kConsumerWarps];
@@ -292,8 +299,8 @@ __device__ __forceinline__ void block_means_any(float *base, uint32_t nblk, uint
 // sample; with MULTI the sum over the samples in ascending order, divided by their
 // number.  hidx indexes the stage's hvp arrays, gidx its Philox groups, j is the
 // element's index in the row (it selects the word and the bit of the signs).
-template <bool MULTI, bool DIST>
-__device__ __forceinline__ float4 hutchinson4(const Stage<DIST> &st, const ExtraSample *xs,
+template <bool MULTI, bool HASC>
+__device__ __forceinline__ float4 hutchinson4(const Stage<HASC> &st, const ExtraSample *xs,
                                               uint32_t nsamp, uint32_t hidx, uint32_t gidx,
                                               uint32_t j, float fn, float rn)
 {
@@ -311,13 +318,14 @@ __device__ __forceinline__ float4 hutchinson4(const Stage<DIST> &st, const Extra
     return D;
 }
 
-template <int POWMODE, bool WD, bool DIST, bool MULTI>
+template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE>
 __global__ void __launch_bounds__(kThreads, MULTI ? 3 : kCtasPerSm)
 local_step_kernel(const __grid_constant__ StepParams p)
 {
+    constexpr bool HASC = DIST || FUSE;            // the stages carry a tile of the master row
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    Shared<DIST> &sh = *reinterpret_cast<Shared<DIST> *>(smem_raw);
-    ExtraSample *extra = reinterpret_cast<ExtraSample *>(smem_raw + sizeof(Shared<DIST>));
+    Shared<HASC> &sh = *reinterpret_cast<Shared<HASC> *>(smem_raw);
+    ExtraSample *extra = reinterpret_cast<ExtraSample *>(smem_raw + sizeof(Shared<HASC>));
     const uint32_t nextra = MULTI ? p.nsamp - 1u : 0u;     // extra samples per stage
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -337,25 +345,33 @@ local_step_kernel(const __grid_constant__ StepParams p)
         uint32_t drawn = 0;
         if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
         uint32_t k = 0;
+        uint32_t tile = 0, r = 0, rows_left = 0;   // FUSE: where the producer is in a tile's worker list
         for (;; ++k) {
             const uint32_t s = k % kStages, use = k / kStages;
             if (use > 0 && !mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout))
                 break;
-            const uint32_t n = __shfl_sync(0xffffffffu, drawn, 0);
-            if (n >= p.nitems) {             // nothing left: tell the consumers and leave
-                if (lane == 0) {
-                    sh.stage[s].flags = kItemEnd;
-                    mbar_arrive(&sh.full[s]);
+            if (!FUSE || rows_left == 0u) {
+                const uint32_t n = __shfl_sync(0xffffffffu, drawn, 0);
+                if (n >= p.nitems) {         // nothing left: tell the consumers and leave
+                    if (lane == 0) {
+                        sh.stage[s].flags = kItemEnd;
+                        mbar_arrive(&sh.full[s]);
+                    }
+                    break;
                 }
-                break;
+                if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
+                if constexpr (FUSE) {
+                    // an item is a tile with all its workers, taken in their arrival order
+                    tile = n; r = 0; rows_left = p.nrows;
+                } else {
+                    // Plain rounds walk one worker's row after the other; distance rounds
+                    // walk the workers innermost, so that a tile of the master row is fetched
+                    // from HBM once and served from L2 to the other workers.
+                    tile = DIST ? n / p.nrows : n % p.ntiles;
+                    r = DIST ? n - tile * p.nrows : n / p.ntiles;
+                }
             }
-            if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
-            Stage<DIST> &st = sh.stage[s];
-            // Plain rounds walk one worker's row after the other; distance rounds walk
-            // the workers innermost, so that a tile of the master row is fetched from
-            // HBM once and served from L2 to the other workers.
-            const uint32_t tile = DIST ? n / p.nrows : n % p.ntiles;
-            const uint32_t r = DIST ? n - tile * p.nrows : n / p.ntiles;
+            Stage<HASC> &st = sh.stage[s];
             const uint32_t i = p.row[r];
             const bool act = p.active[i] != 0;
             const uint32_t t0 = tile * (uint32_t)kTile;
@@ -376,9 +392,12 @@ local_step_kernel(const __grid_constant__ StepParams p)
                                           p.key1, extra[s * nextra + q].zw[lane]);
                 }
             }
+            const bool first = FUSE && r == 0u, last = FUSE && rows_left == 1u;
             if (lane == 0) {
                 st.worker = i; st.t0 = t0; st.nvalid = nvalid;
-                st.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly);
+                st.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly) |
+                           (first ? kItemFirst : 0u) | (last ? kItemLast : 0u) |
+                           (FUSE && p.exch[i] ? kItemExchange : 0u);
                 st.e0 = ti.e0; st.e1 = ti.e1; st.run0 = ti.run0; st.ea0 = ea0;
                 st.tile = tile;
             }
@@ -387,9 +406,10 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 const uint32_t row_bytes = n4 * 4u, hv_bytes = (ea1 - ea0) * 4u;
                 const uint64_t so = (uint64_t)i * p.lds + t0;
                 uint64_t *bar = &sh.full[s];
+                const bool want_c = FUSE ? first : DIST;      // fused: once per tile
                 if (act) {
                     mbar_arrive_expect_tx(bar, 4u * row_bytes + (1u + nextra) * hv_bytes +
-                                                   (DIST ? row_bytes : 0u));
+                                                   (want_c ? row_bytes : 0u));
                     bulk_load(&st.hv[ea0 + kHalo - t0], p.hvp + (uint64_t)i * p.ld + ea0, hv_bytes, bar);
                     if constexpr (MULTI)
                         for (uint32_t q = 0; q < nextra; ++q)
@@ -401,13 +421,14 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     bulk_load(st.x, p.x + so, row_bytes, bar);
                     bulk_load(st.m, p.m + so, row_bytes, bar);
                     bulk_load(st.v, p.v + so, row_bytes, bar);
-                    if constexpr (DIST) bulk_load(st.c, p.c + t0, row_bytes, bar);
-                } else if constexpr (DIST) {
-                    mbar_arrive_expect_tx(bar, 2u * row_bytes);
+                    if constexpr (HASC) if (want_c) bulk_load(st.c, p.c + t0, row_bytes, bar);
+                } else if constexpr (HASC) {
+                    mbar_arrive_expect_tx(bar, (want_c ? 2u : 1u) * row_bytes);
                     bulk_load(st.x, p.x + so, row_bytes, bar);
-                    bulk_load(st.c, p.c + t0, row_bytes, bar);
+                    if (want_c) bulk_load(st.c, p.c + t0, row_bytes, bar);
                 }
             }
+            if constexpr (FUSE) { ++r; --rows_left; }
         }
         // the last producer to leave puts both scheduler words back to zero for the next
         // launch (every producer has made its final fetch before it counts itself out)
@@ -423,16 +444,31 @@ local_step_kernel(const __grid_constant__ StepParams p)
 
     // ================================= consumers =================================
     const int ctid = threadIdx.x;
+    float4 c_old[kPasses], c_acc[kPasses];         // FUSE: carried through the workers of a tile
     uint32_t k = 0;
     for (;; ++k) {
         const uint32_t s = k % kStages, use = k / kStages;
         if (!mbar_wait(&sh.full[s], use & 1u, p.status, kStatusFullTimeout)) break;
-        Stage<DIST> &st = sh.stage[s];
+        Stage<HASC> &st = sh.stage[s];
         const uint32_t i = st.worker, t0 = st.t0, nvalid = st.nvalid, flags = st.flags;
         if (flags & kItemEnd) break;
         const ExtraSample *xs = extra + s * nextra;
         const float fn = (float)p.nsamp, rn = __frcp_rn(fn);
         float4 xn[kPasses];
+        if constexpr (FUSE) {
+            if (flags & kItemFirst) {
+#pragma unroll
+                for (int pass = 0; pass < kPasses; ++pass) {
+                    const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                    if (off < nvalid) {
+                        c_old[pass] = ld_vec(&st.c[off]);
+                        // simultaneous form: what the workers add to the master, from +0;
+                        // asynchronous form: the master as the arrivals so far left it
+                        c_acc[pass] = p.asynchronous ? c_old[pass] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            }
+        }
 
         if (!(flags & kItemDistanceOnly)) {
             const WorkerConst w = p.w[i];
@@ -442,7 +478,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 for (uint32_t q = ctid; q < (ea1 - ea0) >> 2; q += kConsumers) {
                     const uint32_t j = ea0 + 4u * q, hidx = j + kHalo - t0;
                     st_vec(&st.hv[hidx],
-                           hutchinson4<MULTI, DIST>(st, xs, p.nsamp, hidx, (j >> 7) - g0, j, fn, rn));
+                           hutchinson4<MULTI, HASC>(st, xs, p.nsamp, hidx, (j >> 7) - g0, j, fn, rn));
                 }
                 consumer_sync();
                 // ---- block means in place, one thread per block
@@ -471,7 +507,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
                     const float4 D = (flags & kItemAverage)
                         ? ld_vec(&st.hv[off + kHalo])
-                        : hutchinson4<MULTI, DIST>(st, xs, p.nsamp, off + kHalo, off >> 7, off, fn, rn);
+                        : hutchinson4<MULTI, HASC>(st, xs, p.nsamp, off + kHalo, off >> 7, off, fn, rn);
                     const float4 g = ld_vec(&st.g[off]);
                     float4 x = ld_vec(&st.x[off]), m = ld_vec(&st.m[off]), v = ld_vec(&st.v[off]);
                     if (nv == 4) {
@@ -481,13 +517,13 @@ local_step_kernel(const __grid_constant__ StepParams p)
                         if (nv > 1) adahessian_update<POWMODE, WD>(x.y, m.y, v.y, g.y, D.y, p, w);
                         if (nv > 2) adahessian_update<POWMODE, WD>(x.z, m.z, v.z, g.z, D.z, p, w);
                     }
-                    st_vec(xr + off, x);
+                    if constexpr (!FUSE) st_vec(xr + off, x);     // fused: x is stored after the pull
                     st_vec(mr + off, m);
                     st_vec(vr + off, v);
                     xn[pass] = x;
                 }
             }
-        } else if constexpr (DIST) {
+        } else if constexpr (HASC) {
 #pragma unroll
             for (int pass = 0; pass < kPasses; ++pass) {
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
@@ -503,7 +539,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
                 double d = 0.0;
                 if (off < nvalid) {
                     const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
-                    d = dist4(xn[pass], ld_vec(&st.c[off]), nv);
+                    d = dist4(xn[pass], FUSE ? c_old[pass] : ld_vec(&st.c[off]), nv);
                 }
                 d = warp_tree_sum(d);
                 if (lane == 0) red[pass * kConsumerWarps + warp] = d;
@@ -519,6 +555,46 @@ local_step_kernel(const __grid_constant__ StepParams p)
 #pragma unroll
                     for (int q = 0; q < len / 2; ++q) t[q] = __dadd_rn(t[2 * q], t[2 * q + 1]);
                 p.partials[(uint64_t)i * p.ntiles_pad + st.tile] = t[0];
+            }
+        }
+
+        if constexpr (FUSE) {
+            // ---- the elastic pull of this worker against the master (Eqs. 12-13), in the
+            // same operation order as the separate exchange kernels
+            const bool meets = (flags & kItemExchange) != 0u;
+            const float h1 = p.wdev ? p.wdev[p.nworkers + i] : p.h1w[i];
+            const float h2 = p.wdev ? p.wdev[i] : p.h2w[i];
+#pragma unroll
+            for (int pass = 0; pass < kPasses; ++pass) {
+                const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                if (off < nvalid) {
+                    if (meets) {
+                        float *xe = &xn[pass].x, *ae = &c_acc[pass].x;
+                        const float *ce = &c_old[pass].x;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (p.asynchronous) {
+                                const float d = __fsub_rn(xe[e], ae[e]);
+                                xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+                                ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+                            } else {
+                                const float d = __fsub_rn(xe[e], ce[e]);
+                                ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+                                xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+                            }
+                        }
+                    }
+                    if (meets || !(flags & kItemDistanceOnly))
+                        st_vec(p.x + (uint64_t)i * p.lds + t0 + off, xn[pass]);
+                    if ((flags & kItemLast) && p.any_exchange) {
+                        float4 cn = c_acc[pass];
+                        if (!p.asynchronous) {
+                            cn.x = __fadd_rn(c_old[pass].x, cn.x); cn.y = __fadd_rn(c_old[pass].y, cn.y);
+                            cn.z = __fadd_rn(c_old[pass].z, cn.z); cn.w = __fadd_rn(c_old[pass].w, cn.w);
+                        }
+                        st_vec(p.c_out + t0 + off, cn);
+                    }
+                }
             }
         }
 
@@ -632,16 +708,17 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-template <int POWMODE, bool WD, bool DIST, bool MULTI>
+template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE>
 static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream_t s)
 {
-    auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI>;
-    const size_t smem = sizeof(Shared<DIST>) +
+    auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI, FUSE>;
+    constexpr bool HASC = DIST || FUSE;
+    const size_t smem = sizeof(Shared<HASC>) +
                         (MULTI ? (size_t)kStages * (p.nsamp - 1u) * sizeof(ExtraSample) : 0);
     static bool configured = false;      // per instantiation
     static int ctas_for_nsamp[AH_MAX_SAMPLES + 1] = {};
     if (!configured) {
-        const size_t most = sizeof(Shared<DIST>) +
+        const size_t most = sizeof(Shared<HASC>) +
                             (MULTI ? (size_t)kStages * (AH_MAX_SAMPLES - 1) * sizeof(ExtraSample) : 0);
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)most);
@@ -672,11 +749,14 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
 template <int POWMODE, bool WD>
 static cudaError_t launch_step_dist(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
 {
+    if (p.fused)                         // step and exchange in one pass (one Hutchinson sample)
+        return want_dist ? launch_step_one<POWMODE, WD, true, false, true>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, false, true>(p, sm_count, s);
     if (p.nsamp > 1u)
-        return want_dist ? launch_step_one<POWMODE, WD, true, true>(p, sm_count, s)
-                         : launch_step_one<POWMODE, WD, false, true>(p, sm_count, s);
-    return want_dist ? launch_step_one<POWMODE, WD, true, false>(p, sm_count, s)
-                     : launch_step_one<POWMODE, WD, false, false>(p, sm_count, s);
+        return want_dist ? launch_step_one<POWMODE, WD, true, true, false>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, true, false>(p, sm_count, s);
+    return want_dist ? launch_step_one<POWMODE, WD, true, false, false>(p, sm_count, s)
+                     : launch_step_one<POWMODE, WD, false, false, false>(p, sm_count, s);
 }
 
 cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)

@@ -30,6 +30,9 @@ class RunConfig:
     asynchronous: bool = False      # workers reach the master one at a time, seeded order
     sync_free: str = "no"           # "yes": weights on the device (easgd_exchange_dynamic);
                                     # "mixed": device and host forms of the rule alternate
+    fused: str = "no"               # exchange rounds in one pass: "given" (coefficients known
+                                    # before the step: alpha) or "lagged" (the rule's output
+                                    # of the previous exchange round, kept on the device)
     method: str = "adahessian"      # local step: "adahessian", "sgd" or "msgd" (momentum)
     momentum: float = 0.5
     scripted: list = field(default_factory=list)
@@ -62,6 +65,7 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
     alpha = cfg.alpha_value()
     log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "orders_equal": True,
            "exchanges": 0}
+    lagged_weights = None
     for t in range(1, cfg.rounds + 1):
         mask_g = h.dw_mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
         mask_o = ref.mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
@@ -73,6 +77,33 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         common = dict(lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
                       hessian_power=cfg.hessian_power, weight_decay=cfg.weight_decay,
                       want_dist=ex)
+        if cfg.fused != "no" and ex:
+            # one pass: step, distances, pull.  The oracle takes the same steps one by one.
+            log["exchanges"] += 1
+            lag = cfg.fused == "lagged"
+            order_g = order_o = None
+            if cfg.asynchronous:
+                order_g = h.dw_order_next(ORDER_SEED, t)
+                order_o = ref.order_next(ORDER_SEED, t)
+                log["orders_equal"] &= bool(np.array_equal(order_g, order_o))
+            h.ah_local_step_exchange(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
+                                     active=mask_g if cfg.frozen else None, worker_mask=mask_g,
+                                     alpha=alpha, order=order_g, asynchronous=cfg.asynchronous,
+                                     lagged=lag, **dict(common, want_dist=lag or ex))
+            ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
+                           active=mask_o if cfg.frozen else None, **common)
+            h2, h1 = lagged_weights if (lag and lagged_weights is not None) else (None, None)
+            if cfg.asynchronous:
+                ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
+            else:
+                ref.exchange(mask_o, h2, h1, alpha=alpha)
+            log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+            if lag:
+                lagged_weights = ref.weights_next(alpha)            # serves the next exchange round
+                w = h.ah_state_get(binding.AH_WEIGHTS)
+                log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], lagged_weights[0]) and
+                                             np.array_equal(w[cfg.K:], lagged_weights[1]))
+            continue
         if cfg.method == "adahessian":
             h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
                             active=mask_g if cfg.frozen else None, **common)

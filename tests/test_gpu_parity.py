@@ -334,6 +334,86 @@ def test_dynamic_exchange_custom_rule_and_errors(B, torch):
     h.close()
 
 
+# ------------------------------------------- exchange rounds in one pass (fused)
+@pytest.mark.parametrize("layout", ["odd", "resnet18"])
+@pytest.mark.parametrize("asyn", [False, True])
+def test_fused_round_equals_step_then_exchange(B, torch, layout, asyn):
+    if layout == "odd":
+        segs, P = ODD_SEGS, ODD_P
+    else:
+        lay = W.resnet18_layout(16)
+        segs, P = W.segments(lay), W.total_params(lay)
+    K, ld = 5, W.padded_ld(P)
+    rng = np.random.default_rng(70 + P)
+    theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
+    h = B.Handle(K, P, segs)
+    ref = OracleState(theta0, K, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    for t in range(1, 9):
+        g = np.zeros((K, ld), np.float32)
+        hv = np.zeros((K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        hv[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        active = None if t % 3 else (rng.random(K) > 0.4).astype(np.uint8)
+        mask = None if t % 4 == 1 else (rng.random(K) > 0.3).astype(np.uint8)
+        if t == 6:
+            mask = np.zeros(K, np.uint8)                      # nobody meets the master
+        dist = t % 2 == 0
+        order = h.dw_order_next(5, t) if asyn else None
+        if t % 2:
+            h2 = rng.uniform(0, 0.15, K).astype(np.float32)
+            h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+            weights = np.concatenate([h2, h1])
+        else:
+            h2 = h1 = weights = None
+        h.ah_local_step_exchange(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda(), Z_SEED, lr=0.01,
+                                 round_=t, active=active, want_dist=dist, worker_mask=mask,
+                                 weights=weights, alpha=0.1, order=order, asynchronous=asyn)
+        ref.local_step(g, hv, Z_SEED, t, lr=0.01, active=active, want_dist=dist)
+        if asyn:
+            ref.exchange_async(mask, h2, h1, alpha=0.1, order=order)
+        else:
+            ref.exchange(mask, h2, h1, alpha=0.1)
+        if dist:
+            assert np.array_equal(h.ah_state_get(B.AH_NORM2), ref.norm2), t
+        for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v), (B.AH_CENTER, ref.center)):
+            assert np.array_equal(h.ah_state_get(which), want), (t, which)
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    h.close()
+
+
+@pytest.mark.parametrize("asyn,frozen", [(False, False), (True, False), (False, True)])
+def test_fused_rounds_with_lagged_dynamic_weights(B, torch, asyn, frozen):
+    # every exchange round in one pass, the rule's coefficients one period behind the
+    # distances; the oracle takes the same schedule with its separate functions
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=100, tau=2,
+                    p_fail=0.25, max_stale=4 if frozen else 1, frozen=frozen,
+                    alpha=0.1 if asyn else None, asynchronous=asyn, fused="lagged")
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"] and log["orders_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    assert log["exchanges"] == 50
+    h.close()
+
+
+def test_fused_round_argument_checks(B, torch):
+    K, P = 2, 1000
+    h = B.Handle(K, P, [])
+    g = torch.zeros(K, P, device="cuda")
+    with pytest.raises(B.AdaHessError) as e:          # lagged weights need this round's distances
+        h.ah_local_step_exchange(g, g, 1, lr=0.1, lagged=True, want_dist=False)
+    assert e.value.status == B.AH_ERR_INVALID_ARG
+    with pytest.raises(B.AdaHessError) as e:
+        h.ah_local_step_exchange(g, g, 1, lr=0.1, asynchronous=True, order=np.array([1, 1]))
+    assert e.value.status == B.AH_ERR_INVALID_ARG
+    h.close()
+
+
 # ------------------------------------------- first-order local steps (EASGD / EAMSGD)
 @pytest.mark.parametrize("K,P", [(1, 1), (2, 1023), (3, 4097), (4, 184_837), (8, 4 * 1024 * 5), (5, 8193)])
 @pytest.mark.parametrize("delta", [0.0, 0.5])
