@@ -422,7 +422,7 @@ def oracle_periods(args, layout, periods, warm):
                 for r, (g, hv) in enumerate(pool)]
     st = oracle.OracleState(W.theta0_np(layout, DATA_SEED), K, segs, variant="omp")
     alpha = alpha_for(K)
-    t, t_start, worker_steps = 0, None, 0
+    t, t_start, worker_steps, lagged = 0, None, 0, None
     for period in range(warm + periods):
         if period == warm:
             t_start = time.perf_counter()
@@ -439,7 +439,13 @@ def oracle_periods(args, layout, periods, warm):
                 st.sgd_step(g, SGD_LR, SGD_MOMENTUM if args.method == "msgd" else 0.0,
                             active=mask if frozen else None)
             if ex:
-                h2, h1 = st.weights_next(alpha) if args.method == "adahessian" else (None, None)
+                if args.method != "adahessian":
+                    h2, h1 = None, None
+                elif args.fused:     # coefficients one period behind the distances
+                    h2, h1 = lagged if lagged is not None else (None, None)
+                    lagged = st.weights_next(alpha)
+                else:
+                    h2, h1 = st.weights_next(alpha)
                 if args.exchange == "async":
                     st.exchange_async(mask, h2, h1, alpha=alpha, order=st.order_next(ORDER_SEED, t))
                 else:

@@ -641,6 +641,28 @@ def _full_size_run(B, kind, K, tau, rounds, p_fail, max_stale=1, frozen=False, n
     _check_run(B, cfg, _layout_inputs(layout, K, n_pool=n_pool))
 
 
+@pytest.mark.parametrize("variant", ["async_device_weights", "fused_lagged", "fused_lagged_async", "eamsgd"])
+def test_full_size_resnet18_layout_variants(B, torch, variant):
+    # config 2 at its full size with the other forms of the round, in the launch shapes the
+    # bench times: two communication periods each, every element compared with the oracle
+    layout = W.resnet18_layout()
+    kw = dict(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=8, tau=4, p_fail=0.1)
+    if variant == "async_device_weights":
+        cfg = RunConfig(asynchronous=True, sync_free="yes", alpha=0.1, **kw)
+    elif variant == "fused_lagged":
+        cfg = RunConfig(fused="lagged", **kw)
+    elif variant == "fused_lagged_async":
+        cfg = RunConfig(fused="lagged", asynchronous=True, alpha=0.1, **kw)
+    else:
+        cfg = RunConfig(method="msgd", dynamic=False, alpha=0.1, asynchronous=True, **kw)
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8, n_pool=2), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"] and log["orders_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert log["exchanges"] == 2
+    h.close()
+
+
 def test_full_size_resnet18_layout(B, torch):
     # config 2 at its full size (P = 11,689,512, K = 8): two communication periods
     _full_size_run(B, "resnet18", 8, 4, 8, 0.1, n_pool=2)
