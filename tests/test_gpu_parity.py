@@ -335,15 +335,20 @@ def test_dynamic_exchange_custom_rule_and_errors(B, torch):
 
 
 # ------------------------------------------- exchange rounds in one pass (fused)
-@pytest.mark.parametrize("layout", ["odd", "resnet18"])
+@pytest.mark.parametrize("layout", ["odd", "resnet18", "one", "ragged"])
 @pytest.mark.parametrize("asyn", [False, True])
 def test_fused_round_equals_step_then_exchange(B, torch, layout, asyn):
+    K = 5
     if layout == "odd":
         segs, P = ODD_SEGS, ODD_P
+    elif layout == "one":
+        segs, P, K = [], 1, 1                                  # the smallest problem there is
+    elif layout == "ragged":
+        segs, P, K = [(0, 1026, 3)], 2051, 2                   # a block across the tile edge, odd tail
     else:
         lay = W.resnet18_layout(16)
         segs, P = W.segments(lay), W.total_params(lay)
-    K, ld = 5, W.padded_ld(P)
+    ld = W.padded_ld(P)
     rng = np.random.default_rng(70 + P)
     theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
     h = B.Handle(K, P, segs)
