@@ -133,7 +133,8 @@ enum {
                           maximal runs of equal spatial block (get only, host)              */
     AH_TILES = 11,     /* uint32 [tiles][4] {first run, e0, e1, flags}: each tile's range
                           widened to whole spatial blocks [e0, e1); flags bit 0 = the tile
-                          touches a block > 1 (get only, host)                              */
+                          touches a block > 1, bit 1 = every such block is a 3 x 3 kernel
+                          (get only, host)                                                  */
     AH_WEIGHTS = 12    /* float  [2K]  h2[0..K) then h1[0..K) of the last
                           easgd_exchange_dynamic (get only, host)                           */
 };

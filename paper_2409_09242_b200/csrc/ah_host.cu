@@ -111,11 +111,13 @@ void build_tiles(uint32_t P, const std::vector<Run> &runs, std::vector<TileInfo>
         ti.e0 = first.block > 1 ? first.start + (t0 - first.start) / first.block * first.block : t0;
         size_t rj = ri;
         uint32_t flags = 0;
+        bool all9 = true;
         for (;;) {
-            if (runs[rj].block > 1) flags |= 1u;
+            if (runs[rj].block > 1) { flags |= 1u; if (runs[rj].block != 9) all9 = false; }
             if (runs[rj].end >= t1) break;
             ++rj;
         }
+        if ((flags & 1u) && all9) flags |= 2u;
         const Run &last = runs[rj];
         ti.e1 = last.block > 1
                     ? last.start + ((t1 - 1 - last.start) / last.block + 1) * last.block

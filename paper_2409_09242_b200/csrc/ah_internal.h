@@ -61,7 +61,8 @@ struct Run {
 };
 
 // Per tile: first run that intersects it, and the tile's range widened to whole
-// spatial blocks [e0, e1).  flags bit 0: some run with block > 1 intersects the tile.
+// spatial blocks [e0, e1).  flags bit 0: some run with block > 1 intersects the tile;
+// bit 1: every such run has block 9 (3 x 3 kernels), the case with its own fast path.
 struct TileInfo {
     uint32_t run0;
     uint32_t e0;

@@ -226,8 +226,11 @@ __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 // Consumers, per item: wait for the stage; where the tile touches a tensor with
 // spatial block > 1 they turn hvp into z (.) hvp in place, average each block in
 // place (one thread per block, ascending-order sum, one division) and read the
-// means back; otherwise the sign is applied in registers.  Then moments and update
-// per element, 128-bit stores of x, m, v, and the stage goes back to the producer.
+// means back; otherwise the sign is applied in registers.  Tiles whose averaged
+// tensors are all 3 x 3 kernels (the common case) skip the separate sign pass: the
+// thread that sums a block takes the nine signs from the Philox words as it goes.
+// Then moments and update per element, 128-bit stores of x, m, v, and the stage goes
+// back to the producer.
 //
 // DIST additionally leaves, per tile, the pairwise-tree sum of (x_new - c)^2 in
 // p.partials[worker][tile], for every worker; a worker that sits the step out
@@ -240,6 +243,7 @@ enum : uint32_t {
     kItemFirst = 8u,          // fused exchange: first worker of a tile (c was fetched with it)
     kItemLast = 16u,          // fused exchange: last worker of a tile (the master is written back)
     kItemExchange = 32u,      // fused exchange: this worker meets the master
+    kItemAll3x3 = 64u,        // every averaged tensor the tile touches has block 9
 };
 
 template <bool HASC>
@@ -280,6 +284,35 @@ __device__ __forceinline__ void block_means_fixed(float *base, uint32_t nblk, in
         const float mean = div_by_const(S, fb, rb);
 #pragma unroll
         for (int e = 0; e < B; ++e) blk[e] = mean;
+    }
+}
+
+// Block means of 3x3 kernels straight from the raw Hessian-vector values: the signs
+// of the nine elements are taken from the Philox words on the fly.
+template <bool HASC>
+__device__ __forceinline__ void block_means_signed9(Stage<HASC> &st, uint32_t qa, uint32_t nblk,
+                                                    uint32_t t0, uint32_t g0, int ctid)
+{
+    const float rb = __frcp_rn(9.0f);
+    for (uint32_t k = ctid; k < nblk; k += kConsumers) {
+        const uint32_t j0 = qa + 9u * k;
+        float *blk = &st.hv[j0 + kHalo - t0];
+        const uint32_t w0 = j0 >> 5, w1 = (j0 + 8u) >> 5;       // words holding the first and last sign
+        const uint32_t lo = st.zw[(w0 >> 2) - g0][w0 & 3u];
+        const uint32_t hi = st.zw[(w1 >> 2) - g0][w1 & 3u];     // == lo when the block sits in one word
+        const uint32_t bits = __funnelshift_r(lo, hi, j0 & 31u);
+        float S = flip_if_bit<0>(blk[0], bits);
+        S = __fadd_rn(S, flip_if_bit<1>(blk[1], bits));
+        S = __fadd_rn(S, flip_if_bit<2>(blk[2], bits));
+        S = __fadd_rn(S, flip_if_bit<3>(blk[3], bits));
+        S = __fadd_rn(S, flip_if_bit<4>(blk[4], bits));
+        S = __fadd_rn(S, flip_if_bit<5>(blk[5], bits));
+        S = __fadd_rn(S, flip_if_bit<6>(blk[6], bits));
+        S = __fadd_rn(S, flip_if_bit<7>(blk[7], bits));
+        S = __fadd_rn(S, flip_if_bit<8>(blk[8], bits));
+        const float mean = div_by_const(S, 9.0f, rb);
+#pragma unroll
+        for (int e = 0; e < 9; ++e) blk[e] = mean;
     }
 }
 
@@ -396,6 +429,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
             if (lane == 0) {
                 st.worker = i; st.t0 = t0; st.nvalid = nvalid;
                 st.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly) |
+                           ((ti.flags & 2u) ? kItemAll3x3 : 0u) |
                            (first ? kItemFirst : 0u) | (last ? kItemLast : 0u) |
                            (FUSE && p.exch[i] ? kItemExchange : 0u);
                 st.e0 = ti.e0; st.e1 = ti.e1; st.run0 = ti.run0; st.ea0 = ea0;
@@ -473,29 +507,50 @@ local_step_kernel(const __grid_constant__ StepParams p)
         if (!(flags & kItemDistanceOnly)) {
             const WorkerConst w = p.w[i];
             if (flags & kItemAverage) {
-                // ---- z (.) hvp in place over the widened range
                 const uint32_t ea0 = st.ea0, ea1 = (st.e1 + 3u) & ~3u, g0 = ea0 >> 7;
-                for (uint32_t q = ctid; q < (ea1 - ea0) >> 2; q += kConsumers) {
-                    const uint32_t j = ea0 + 4u * q, hidx = j + kHalo - t0;
-                    st_vec(&st.hv[hidx],
-                           hutchinson4<MULTI, HASC>(st, xs, p.nsamp, hidx, (j >> 7) - g0, j, fn, rn));
-                }
-                consumer_sync();
-                // ---- block means in place, one thread per block
                 const uint32_t e0 = st.e0, e1 = st.e1;
-                for (uint32_t ri = st.run0;; ++ri) {
-                    const Run rn = p.runs[ri];
-                    if (rn.start >= e1) break;
-                    if (rn.block > 1u) {
+                if (!MULTI && (flags & kItemAll3x3)) {
+                    // ---- 3x3 kernels only: means from the raw values, signs on the fly;
+                    // ranges of unaveraged tensors inside the tile get their signs in place
+                    for (uint32_t ri = st.run0;; ++ri) {
+                        const Run rn = p.runs[ri];
+                        if (rn.start >= e1) break;
                         const uint32_t qa = max(e0, rn.start), qb = min(e1, rn.end);
-                        const uint32_t nblk = __umulhi(qb - qa, rn.magic);
-                        float *base = &st.hv[qa + kHalo - t0];
-                        if (rn.block == 9u) block_means_fixed<9>(base, nblk, ctid);
-                        else block_means_any(base, nblk, rn.block, ctid);
+                        if (rn.block > 1u) {
+                            block_means_signed9(st, qa, __umulhi(qb - qa, rn.magic), t0, g0, ctid);
+                        } else {
+                            for (uint32_t j = qa + ctid; j < qb; j += kConsumers) {
+                                const uint32_t word = st.zw[(j >> 7) - g0][(j >> 5) & 3u];
+                                float *ptr = &st.hv[j + kHalo - t0];
+                                *ptr = __uint_as_float(__float_as_uint(*ptr) ^ (((word >> (j & 31u)) & 1u) << 31));
+                            }
+                        }
+                        if (rn.end >= e1) break;
                     }
-                    if (rn.end >= e1) break;
+                    consumer_sync();
+                } else {
+                    // ---- z (.) hvp in place over the widened range
+                    for (uint32_t q = ctid; q < (ea1 - ea0) >> 2; q += kConsumers) {
+                        const uint32_t j = ea0 + 4u * q, hidx = j + kHalo - t0;
+                        st_vec(&st.hv[hidx],
+                               hutchinson4<MULTI, HASC>(st, xs, p.nsamp, hidx, (j >> 7) - g0, j, fn, rn));
+                    }
+                    consumer_sync();
+                    // ---- block means in place, one thread per block
+                    for (uint32_t ri = st.run0;; ++ri) {
+                        const Run rn = p.runs[ri];
+                        if (rn.start >= e1) break;
+                        if (rn.block > 1u) {
+                            const uint32_t qa = max(e0, rn.start), qb = min(e1, rn.end);
+                            const uint32_t nblk = __umulhi(qb - qa, rn.magic);
+                            float *base = &st.hv[qa + kHalo - t0];
+                            if (rn.block == 9u) block_means_fixed<9>(base, nblk, ctid);
+                            else block_means_any(base, nblk, rn.block, ctid);
+                        }
+                        if (rn.end >= e1) break;
+                    }
+                    consumer_sync();
                 }
-                consumer_sync();
             }
             float *xr = p.x + (uint64_t)i * p.lds + t0;
             float *mr = p.m + (uint64_t)i * p.lds + t0;

@@ -153,7 +153,10 @@ def test_tile_descriptors_cover_whole_blocks(B, name):
         assert runs[run0, 0] <= t0 < runs[run0, 1]
         assert e0 <= t0 and e1 >= t1 and e1 <= P
         assert t0 - e0 < B.AH_MAX_BLOCK and e1 - t1 < B.AH_MAX_BLOCK
-        assert flags == int(np.any(block_of[t0:t1] > 1))
+        averaged = block_of[t0:t1][block_of[t0:t1] > 1]
+        assert flags & 1 == int(averaged.size > 0)
+        assert (flags >> 1) & 1 == int(averaged.size > 0 and np.all(averaged == 9))   # 3x3 kernels only
+        assert flags >> 2 == 0
         # [e0, e1) ends on block boundaries of the runs they fall in
         for edge in (e0, e1):
             r = np.searchsorted(runs[:, 1], edge, side="right" if edge == e0 else "left")
