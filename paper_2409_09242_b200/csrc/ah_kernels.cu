@@ -352,7 +352,7 @@ __device__ __forceinline__ float4 hutchinson4(const Stage<HASC> &st, const Extra
 }
 
 template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE>
-__global__ void __launch_bounds__(kThreads, MULTI ? 3 : kCtasPerSm)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 local_step_kernel(const __grid_constant__ StepParams p)
 {
     constexpr bool HASC = DIST || FUSE;            // the stages carry a tile of the master row
