@@ -230,7 +230,9 @@ int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *h
  *   lagged == 0: weights (host, 2K floats: h2 then h1) or, when NULL, alpha for all;
  *   lagged != 0: the dynamic rule of Sec. V-B runs on the device after this round's
  *       distances (hy->want_dist must be 1, weights NULL) and its coefficients serve the
- *       NEXT lagged round; the first lagged round of a handle uses alpha.  This is the
+ *       NEXT lagged round: a lagged round pulls with the most recent output of the rule on
+ *       the device (from an earlier lagged round or from easgd_exchange_dynamic), or with
+ *       alpha while the rule has not yet run there.  This is the
  *       paper's "estimate of the master model": the score follows the distances with a
  *       delay of one communication period, and no call waits for the GPU.
  * One Hutchinson sample per step.  Memory traffic: 32 bytes per parameter update plus 8

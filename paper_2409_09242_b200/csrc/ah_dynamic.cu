@@ -43,6 +43,7 @@ int ah::enqueue_weight_rule(ah_ctx *h, float alpha)
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
     h->launches += 1;
     h->norm2_pending = false;                      // these distances have fed the rule
+    h->lagged_ready = true;                        // weights_dev now holds coefficients
     return AH_OK;
 }
 

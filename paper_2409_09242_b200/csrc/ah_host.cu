@@ -426,7 +426,6 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         if (fx && fx->lagged) {                   // the rule runs now, its output serves next time
             const int rc2 = enqueue_weight_rule(h, fx->alpha);
             if (rc2 != AH_OK) return rc2;
-            h->lagged_ready = true;
         }
     }
     return AH_OK;
