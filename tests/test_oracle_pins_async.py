@@ -189,3 +189,29 @@ def test_order_is_uniform_over_permutations(orc):
         o = orc.order_next(16, 999, t)
         pos[o, np.arange(16)] += 1
     assert np.abs(pos - 500).max() < 5 * math.sqrt(500)
+
+
+# ------------------------------------------------------------------ OpenMP build
+def test_openmp_build_is_bit_identical_for_the_newer_steps():
+    # the parity tests time-box themselves by using the OpenMP build of the oracle: it must
+    # give the single-thread build's bits for the asynchronous exchange, the first-order
+    # steps, several Hutchinson samples and the partition as well
+    import oracle
+    results = []
+    for variant in ("fp32", "omp"):
+        rng = np.random.default_rng(90)
+        K, P, segs = 5, 700, [(0, 630, 9), (640, 49, 49)]
+        st = OracleState(rng.standard_normal(P).astype(np.float32), K, segs, variant=variant)
+        for t in range(1, 9):
+            g = rng.standard_normal((K, P)).astype(np.float32)
+            hv = rng.standard_normal((3, K, P)).astype(np.float32)
+            if t % 2:
+                st.local_step(g, hv, 11, t, lr=0.01, want_dist=True)
+            else:
+                st.sgd_step(g, 0.01, 0.5, active=(rng.random(K) > 0.3).astype(np.uint8), want_dist=True)
+            h2, h1 = st.weights_next(0.1)
+            st.exchange_async((rng.random(K) > 0.3).astype(np.uint8), h2, h1, order=st.order_next(3, t))
+        perm, bounds = oracle.load(variant).partition(17, 5000, 7, 600)
+        results.append((st.x.copy(), st.m.copy(), st.v.copy(), st.center.copy(), st.uhist.copy(), perm, bounds))
+    for a, b in zip(*results):
+        assert np.array_equal(a, b)
