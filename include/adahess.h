@@ -23,7 +23,8 @@
  *     reused as soon as it returns.
  *   - All kernels are enqueued on the handle's stream and the calls return without
  *     waiting, except where a function is marked "synchronises".
- *   - A handle must not be used from two threads at once.
+ *   - A handle must not be used from two threads at once.  The handle's CUDA device
+ *     must be the calling thread's current device for every call after ah_init.
  *   - Arithmetic: IEEE binary32, round-to-nearest, one rounding per operation in
  *     the order the formulas below are written (no fused multiply-add).
  */

@@ -9,6 +9,8 @@
 // Arithmetic follows one fixed order with one binary32 rounding per operation
 // (__fmul_rn / __fadd_rn / __fdiv_rn / __fsqrt_rn are never contracted into FMAs),
 // so results do not depend on compiler flags or launch shape.
+#include <atomic>
+
 #include "ah_internal.h"
 #include "ah_device.cuh"
 
@@ -770,9 +772,14 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
     constexpr bool HASC = DIST || FUSE;
     const size_t smem = sizeof(Shared<HASC>) +
                         (MULTI ? (size_t)kStages * (p.nsamp - 1u) * sizeof(ExtraSample) : 0);
-    static bool configured = false;      // per instantiation
-    static int ctas_for_nsamp[AH_MAX_SAMPLES + 1] = {};
-    if (!configured) {
+    // Shared-memory attributes are per device and per instantiation: one bit per device
+    // ordinal.  Setting them twice is harmless, so racing threads need no lock.
+    static std::atomic<uint64_t> configured{0};
+    static std::atomic<int> ctas_for_nsamp[AH_MAX_SAMPLES + 1] = {};
+    int device = 0;
+    if (cudaError_t e = cudaGetDevice(&device); e != cudaSuccess) return e;
+    const uint64_t device_bit = 1ull << (device & 63);
+    if (!(configured.load(std::memory_order_acquire) & device_bit)) {
         const size_t most = sizeof(Shared<HASC>) +
                             (MULTI ? (size_t)kStages * (AH_MAX_SAMPLES - 1) * sizeof(ExtraSample) : 0);
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -781,19 +788,19 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.fetch_or(device_bit, std::memory_order_release);
     }
     if (p.nitems == 0) return cudaSuccess;
     int ctas = kCtasPerSm;
     if (MULTI) {                         // the extra samples decide how many CTAs fit
-        if (ctas_for_nsamp[p.nsamp] == 0) {
+        if (ctas_for_nsamp[p.nsamp].load(std::memory_order_relaxed) == 0) {
             int fit = 0;
             cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, kThreads, smem);
             if (e != cudaSuccess) return e;
             if (fit < 1) return cudaErrorInvalidConfiguration;
-            ctas_for_nsamp[p.nsamp] = fit;
+            ctas_for_nsamp[p.nsamp].store(fit, std::memory_order_relaxed);
         }
-        ctas = ctas_for_nsamp[p.nsamp];
+        ctas = ctas_for_nsamp[p.nsamp].load(std::memory_order_relaxed);
     }
     const uint32_t resident = (uint32_t)sm_count * (uint32_t)ctas;
     const uint32_t grid = p.nitems < resident ? p.nitems : resident;
