@@ -673,6 +673,11 @@ def test_full_size_resnet18_layout(B, torch):
     _full_size_run(B, "resnet18", 8, 4, 8, 0.1, n_pool=2)
 
 
+def test_full_size_resnet18_layout_all_200_rounds(B, torch):
+    # config 2 exactly as stated: full size, K = 8, tau = 4, Bernoulli(0.1) failures, 200 rounds
+    _full_size_run(B, "resnet18", 8, 4, 200, 0.1, n_pool=2)
+
+
 def test_full_size_resnet50_layout_stragglers(B, torch):
     # config 3 at its full size (P = 25,557,032, K = 16), frozen stragglers
     _full_size_run(B, "resnet50", 16, 4, 4, 0.2, max_stale=8, frozen=True)
