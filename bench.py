@@ -146,11 +146,13 @@ def whole_job_updates_per_second(updates_per_rank, world, ms):
 
 
 def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
-               method="adahessian", sync_free=False, fused=False):
+               method="adahessian", sync_free=False, fused=False, carry=None):
     """One communication period starting after round t0.  With `stage` = (host_pool,
     dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
-    memory (the end-to-end leg).  Returns (next t0, worker-steps taken, workers that
-    exchanged)."""
+    memory (the end-to-end leg).  With `carry` (a dict kept by the caller) the exchange
+    of a period is not launched at its end but rides on the first local step of the next
+    period (one pass over x instead of two, same result).  Returns (next t0, worker-steps
+    taken, workers that exchanged)."""
     import torch
     _, K, tau, p_fail, max_stale, frozen = wl
     alpha = alpha_for(K)
@@ -171,9 +173,16 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
         first_order = method != "adahessian"     # EASGD / EAMSGD: fixed alpha, no distances
+        rode = False
         if first_order:
             h.sgd_local_step(g, SGD_LR, SGD_MOMENTUM if method == "msgd" else 0.0,
                              active=mask if frozen else None)
+        elif carry is not None and carry.get("pending") is not None:
+            rode = True
+            p_mask, p_order = carry.pop("pending")
+            h.easgd_exchange_then_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None,
+                                       worker_mask=p_mask, alpha=alpha, order=p_order,
+                                       asynchronous=asynchronous, dynamic=True, **HYPER)
         elif fused and ex:
             # the whole exchange round in one pass; the rule's coefficients lag one period
             h.ah_local_step_exchange(g, hv, Z_SEED, round_=t, active=mask if frozen else None,
@@ -187,8 +196,11 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         worker_steps += n_act
         if events is not None:
             e1.record()
-            events.append((e0, e1, ex, n_act))
-        if ex and fused and not first_order:
+            events.append((e0, e1, 2 if rode else int(ex), n_act))
+        if ex and carry is not None and not first_order:
+            carry["pending"] = (mask, h.dw_order_next(ORDER_SEED, t) if asynchronous else None)
+            exchanged += int(mask.sum())
+        elif ex and fused and not first_order:
             exchanged += int(mask.sum())
         elif ex:
             on_device = sync_free and not first_order      # weights computed on the device
@@ -253,8 +265,13 @@ def gpu_arm(args):
 
     t = 0
     asyn = args.exchange == "async"
+    # with a period of one round every step also measures distances, which cannot ride along
+    ride = (args.exchange_pass == "next-step" and args.method == "adahessian" and not args.fused
+            and tau >= 2)
+    carry = {} if ride else None
     for _ in range(args.warmup):
-        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused)
+        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused,
+                             carry=carry)
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -266,12 +283,18 @@ def gpu_arm(args):
     worker_steps = exchanged = 0
     for _ in range(args.steps):
         t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events,
-                                method=args.method, sync_free=args.sync_free, fused=args.fused)
+                                method=args.method, sync_free=args.sync_free, fused=args.fused,
+                                carry=carry)
         worker_steps += ws
         exchanged += exd
     stop.record()
     barrier()
     ms = start.elapsed_time(stop)
+    if carry is not None and carry.get("pending") is not None:
+        # the last timed period's exchange would ride on the next step; the first timed
+        # period carried the one before it.  Launch it now, outside the timed region.
+        p_mask, p_order = carry.pop("pending")
+        h.easgd_exchange_dynamic(p_mask, alpha_for(K), p_order, asyn)
     clocks = sampler.stop() if rank == 0 else None
     launches = h.ah_launch_count() - launches0
     ms = max_over_ranks(ms, dist, dev)
@@ -280,8 +303,9 @@ def gpu_arm(args):
 
     # per-launch duration of the fused local-step kernel (plain rounds; the rounds that
     # also measure distances are listed beside it)
-    plain = [(a.elapsed_time(b), n) for a, b, ex, n in events if not ex]
-    withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex]
+    plain = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex == 0]
+    withd = [(a.elapsed_time(b), n) for a, b, ex, n in events if ex == 1]
+    rides = [a.elapsed_time(b) for a, b, ex, n in events if ex == 2]
     # algorithmic bytes of a launch: 32 per update; a distance round also reads the
     # master row once and the x of every worker that sat the step out
     bpu = {"adahessian": 28 + 4 * args.samples, "sgd": 12, "msgd": 20}[args.method]
@@ -305,9 +329,10 @@ def gpu_arm(args):
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": traffic,
                 "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
-                "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None}
+                "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None,
+                "exchange_plus_step_ms": round(sum(rides) / len(rides), 4) if rides else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
-    if args.fused and args.method == "adahessian":
+    if (args.fused or ride) and args.method == "adahessian":
         # fused exchange rounds: x crosses HBM once; the master row is read and written once
         run_bytes = bpu * P * worker_steps + 8 * P * args.steps
     else:
@@ -366,6 +391,7 @@ def gpu_arm(args):
                                   "msgd": "SGD with momentum 0.5, fixed alpha (EAMSGD)"}[args.method],
                    "hutchinson_samples": args.samples,
                    "exchange_rounds": "one pass (step + pull), weights one period behind" if args.fused
+                                      else "the exchange rides on the next round's local step" if ride
                                       else "local step, then exchange kernel",
                    "weights": "on the device, no host wait" if args.sync_free else "on the host, one wait per period",
                    "rounds_timed": tau * args.steps, "input_pool": n_pool,
@@ -504,6 +530,9 @@ def main():
     ap.add_argument("--host-weights", dest="sync_free", action="store_false",
                     help="dynamic weights computed on the host (one wait per period) instead of "
                          "on the device; same bits either way")
+    ap.add_argument("--exchange-pass", default="next-step", choices=["next-step", "separate"],
+                    help="the exchange rides on the next round's local step (one pass over x, same "
+                         "bits), or runs as a kernel of its own")
     ap.add_argument("--fused", action="store_true",
                     help="exchange rounds in one pass (step + pull), dynamic weights one period behind")
     ap.add_argument("--samples", type=int, default=1, help="Hutchinson samples per step (paper: 1)")

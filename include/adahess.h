@@ -244,6 +244,26 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
                            const float *weights, float alpha, const uint16_t *order,
                            int asynchronous, int lagged);
 
+/* The exchange of the round just finished and the local step of the next round in one
+ * pass: tile by tile, each worker first meets the master (easgd_exchange, or
+ * easgd_exchange_async with `order` when asynchronous != 0) and then takes its local
+ * step (ah_local_step) on the pulled parameters.  Bit for bit the result of the two
+ * calls in sequence; x is read and written once instead of twice.  Unlike
+ * ah_local_step_exchange nothing lags: the coefficients are those of this exchange,
+ *   dynamic == 0: weights (host, 2K floats) or, when NULL, alpha for all;
+ *   dynamic != 0: the rule of Sec. V-B runs on the device first, on the distances the
+ *       last want_dist step left there (as easgd_exchange_dynamic; weights must be NULL;
+ *       STATE if no distances are pending), and the pass reads its output.
+ * worker_mask says who takes part in the exchange; hy->active who takes the step.
+ * hy->want_dist must be 0 (the distances to the new master are only defined once every
+ * worker has met it) and hy->n_samples at most 1: with a communication period of one
+ * round use ah_local_step_exchange or the separate calls.  Nothing waits for the GPU.
+ * Errors: INVALID_ARG, ALIGN, STATE, CUDA. */
+int easgd_exchange_then_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
+                             uint64_t z_seed, const ah_hyper *hy, const uint8_t *worker_mask,
+                             const float *weights, float alpha, const uint16_t *order,
+                             int asynchronous, int dynamic);
+
 /* Parameters of the dynamic weighting rule (Sec. V-B): history depth p, the
  * coefficients c_0..c_{p-1} of Eqs. 10-11 (c_0 weighs the newest difference; they
  * should sum to 1) and the threshold kappa < 0 of h1/h2.  Defaults set by ah_init:

@@ -34,7 +34,7 @@ AH_DEVICE_NONE = -2
 
 EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_state_get",
            "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step",
-           "ah_local_step_exchange", "dw_config",
+           "ah_local_step_exchange", "easgd_exchange_then_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
            "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
@@ -74,6 +74,7 @@ _lib.ah_sample_z.argtypes = [_vp, C.c_uint64, C.c_uint32, _vp, C.c_uint64]
 _lib.ah_local_step_exchange.argtypes = [_vp, _vp, _vp, C.c_uint64, C.c_uint64, C.POINTER(ah_hyper),
                                         C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
                                         C.POINTER(C.c_uint16), C.c_int, C.c_int]
+_lib.easgd_exchange_then_step.argtypes = _lib.ah_local_step_exchange.argtypes
 _lib.ah_sample_z_n.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_uint32, _vp, C.c_uint64]
 _lib.ah_local_step.argtypes = [_vp, _vp, _vp, C.c_uint64, C.c_uint64, C.POINTER(ah_hyper)]
 _lib.dw_config.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), C.c_double]
@@ -362,6 +363,37 @@ class Handle:
                                                 grad.stride(0), int(z_seed), C.byref(hy), m, w, alpha, o,
                                                 1 if asynchronous else 0, 1 if lagged else 0),
                     "ah_local_step_exchange")
+
+    def easgd_exchange_then_step(self, grad, hvp, z_seed, lr, beta1=0.9, beta2=0.999, eps=1e-4,
+                                 hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
+                                 worker_mask=None, weights=None, alpha=0.0, order=None,
+                                 asynchronous=False, dynamic=False):
+        if grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
+            raise ValueError("grad and hvp must share shape and row stride")
+        act = m = w = o = None
+        if active is not None:
+            act = np.ascontiguousarray(active, np.uint8)
+            if act.size != self.K:
+                raise ValueError("active: K bytes")
+        if worker_mask is not None:
+            worker_mask = np.ascontiguousarray(worker_mask, np.uint8)
+            m = worker_mask.ctypes.data_as(C.POINTER(C.c_uint8))
+        if weights is not None:
+            weights = np.ascontiguousarray(weights, np.float32)
+            if weights.size != 2 * self.K:
+                raise ValueError("weights: 2K floats (h2 then h1)")
+            w = weights.ctypes.data_as(C.POINTER(C.c_float))
+        if order is not None:
+            order = np.ascontiguousarray(order, np.uint16)
+            if order.size != self.K:
+                raise ValueError("order: K entries")
+            o = order.ctypes.data_as(C.POINTER(C.c_uint16))
+        hy = ah_hyper(lr, beta1, beta2, eps, hessian_power, weight_decay, int(round_),
+                      act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None, 0, 1, 0)
+        self._check(_lib.easgd_exchange_then_step(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
+                                                  grad.stride(0), int(z_seed), C.byref(hy), m, w, alpha,
+                                                  o, 1 if asynchronous else 0, 1 if dynamic else 0),
+                    "easgd_exchange_then_step")
 
     def dw_config(self, p_hist, c, kappa):
         c = np.ascontiguousarray(c, np.float64)

@@ -343,6 +343,9 @@ struct FusedExchange {
     const uint16_t *order;    // host, K entries, or null (ascending)
     bool asynchronous;
     bool lagged;              // coefficients come from the device (previous round's rule)
+    bool before_step;         // the exchange precedes the local step (it belongs to the
+                              // previous round); coefficients from the device if `dynamic`
+    bool dynamic;             // run the rule on the pending distances first
 };
 
 int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
@@ -382,16 +385,22 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     p.eps = hy->eps; p.hpow = hy->hessian_power; p.wd = hy->weight_decay;
     p.fused = fx ? 1u : 0u;
     p.asynchronous = fx && fx->asynchronous ? 1u : 0u;
+    p.pull_first = fx && fx->before_step ? 1u : 0u;
     p.any_exchange = 0u;
     p.nworkers = (uint32_t)h->K;
     p.c_out = h->c;
-    p.wdev = fx && fx->lagged && h->lagged_ready ? h->weights_dev : nullptr;
+    p.wdev = fx && ((fx->lagged && h->lagged_ready) || fx->dynamic) ? h->weights_dev : nullptr;
     if (fx && fx->order) {                        // must name every worker exactly once
         bool seen[AH_MAX_WORKERS] = {};
         for (int q = 0; q < h->K; ++q) {
             if (fx->order[q] >= h->K || seen[fx->order[q]]) return AH_ERR_INVALID_ARG;
             seen[fx->order[q]] = true;
         }
+    }
+    if (fx && fx->dynamic) {                      // this exchange's coefficients, on the device
+        if (!h->norm2_pending) return AH_ERR_STATE;
+        const int rc = enqueue_weight_rule(h, fx->alpha);
+        if (rc != AH_OK) return rc;
     }
     h->calls += 1;
     p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
@@ -450,6 +459,22 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
     FusedExchange fx;
     fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;
     fx.asynchronous = asynchronous != 0; fx.lagged = lagged != 0;
+    fx.before_step = false; fx.dynamic = false;
+    return local_step_impl(h, grad, hvp, ld, z_seed, hy, &fx);
+}
+
+int easgd_exchange_then_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
+                             uint64_t z_seed, const ah_hyper *hy, const uint8_t *worker_mask,
+                             const float *weights, float alpha, const uint16_t *order,
+                             int asynchronous, int dynamic)
+{
+    if (!hy) return AH_ERR_INVALID_ARG;
+    if (hy->n_samples > 1 || hy->want_dist) return AH_ERR_INVALID_ARG;
+    if (dynamic && weights) return AH_ERR_INVALID_ARG;
+    FusedExchange fx;
+    fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;
+    fx.asynchronous = asynchronous != 0; fx.lagged = false;
+    fx.before_step = true; fx.dynamic = dynamic != 0;
     return local_step_impl(h, grad, hvp, ld, z_seed, hy, &fx);
 }
 

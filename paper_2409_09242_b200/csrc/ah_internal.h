@@ -103,6 +103,7 @@ struct StepParams {
     // fused step + exchange (one pass on exchange rounds); unused otherwise
     uint32_t fused;                   // 1: an item is a tile with all its workers, in row order
     uint32_t asynchronous;            // 1: workers meet the master one at a time, in row order
+    uint32_t pull_first;              // 1: a worker meets the master before its local step
     uint32_t any_exchange;            // 0: nobody meets the master, it is not written
     uint32_t nworkers;                // K, for the layout of wdev
     float *c_out;                     // the master row, written once per tile

@@ -330,6 +330,29 @@ __device__ __forceinline__ void block_means_any(float *base, uint32_t nblk, uint
     }
 }
 
+// One worker meets the master on four consecutive columns (Eqs. 12-13), in the operation
+// order of the separate exchange kernels.  Simultaneous form: every worker sees the old
+// master value c_old and `carry` gathers what the workers add to it, from +0.
+// Asynchronous form: `carry` is the master as the arrivals so far left it.
+__device__ __forceinline__ void meet_master4(float4 &x, float4 &carry, const float4 &c_old, float h1,
+                                             float h2, bool asynchronous)
+{
+    float *xe = &x.x, *ae = &carry.x;
+    const float *ce = &c_old.x;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if (asynchronous) {
+            const float d = __fsub_rn(xe[e], ae[e]);
+            xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+            ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+        } else {
+            const float d = __fsub_rn(xe[e], ce[e]);
+            ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+            xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+        }
+    }
+}
+
 // Hutchinson estimate of four consecutive elements (Sec. IV-B): z (.) hvp for one
 // sample; with MULTI the sum over the samples in ascending order, divided by their
 // number.  hidx indexes the stage's hvp arrays, gidx its Philox groups, j is the
@@ -491,6 +514,15 @@ local_step_kernel(const __grid_constant__ StepParams p)
         const ExtraSample *xs = extra + s * nextra;
         const float fn = (float)p.nsamp, rn = __frcp_rn(fn);
         float4 xn[kPasses];
+        // fused exchange: does this worker meet the master, with which coefficients, and
+        // before its local step (the exchange of the previous round) or after it
+        const bool meets = FUSE && (flags & kItemExchange) != 0u;
+        const bool meets_first = meets && p.pull_first != 0u;
+        float h1 = 0.f, h2 = 0.f;
+        if constexpr (FUSE) {
+            h1 = p.wdev ? p.wdev[p.nworkers + i] : p.h1w[i];
+            h2 = p.wdev ? p.wdev[i] : p.h2w[i];
+        }
         if constexpr (FUSE) {
             if (flags & kItemFirst) {
 #pragma unroll
@@ -567,6 +599,9 @@ local_step_kernel(const __grid_constant__ StepParams p)
                         : hutchinson4<MULTI, HASC>(st, xs, p.nsamp, off + kHalo, off >> 7, off, fn, rn);
                     const float4 g = ld_vec(&st.g[off]);
                     float4 x = ld_vec(&st.x[off]), m = ld_vec(&st.m[off]), v = ld_vec(&st.v[off]);
+                    if constexpr (FUSE)
+                        if (meets_first)
+                            meet_master4(x, c_acc[pass], c_old[pass], h1, h2, p.asynchronous != 0u);
                     if (nv == 4) {
                         adahessian_update4<POWMODE, WD>(x, m, v, g, D, p, w);
                     } else {     // ragged end of the row: lanes past P keep their (zero) state
@@ -584,7 +619,12 @@ local_step_kernel(const __grid_constant__ StepParams p)
 #pragma unroll
             for (int pass = 0; pass < kPasses; ++pass) {
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
-                if (off < nvalid) xn[pass] = ld_vec(&st.x[off]);
+                if (off < nvalid) {
+                    xn[pass] = ld_vec(&st.x[off]);
+                    if constexpr (FUSE)
+                        if (meets_first)
+                            meet_master4(xn[pass], c_acc[pass], c_old[pass], h1, h2, p.asynchronous != 0u);
+                }
             }
         }
 
@@ -616,31 +656,13 @@ local_step_kernel(const __grid_constant__ StepParams p)
         }
 
         if constexpr (FUSE) {
-            // ---- the elastic pull of this worker against the master (Eqs. 12-13), in the
-            // same operation order as the separate exchange kernels
-            const bool meets = (flags & kItemExchange) != 0u;
-            const float h1 = p.wdev ? p.wdev[p.nworkers + i] : p.h1w[i];
-            const float h2 = p.wdev ? p.wdev[i] : p.h2w[i];
+            // ---- the elastic pull after the step, the stores of x, and the master row
 #pragma unroll
             for (int pass = 0; pass < kPasses; ++pass) {
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
                 if (off < nvalid) {
-                    if (meets) {
-                        float *xe = &xn[pass].x, *ae = &c_acc[pass].x;
-                        const float *ce = &c_old[pass].x;
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if (p.asynchronous) {
-                                const float d = __fsub_rn(xe[e], ae[e]);
-                                xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
-                                ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
-                            } else {
-                                const float d = __fsub_rn(xe[e], ce[e]);
-                                ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
-                                xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
-                            }
-                        }
-                    }
+                    if (meets && !meets_first)
+                        meet_master4(xn[pass], c_acc[pass], c_old[pass], h1, h2, p.asynchronous != 0u);
                     if (meets || !(flags & kItemDistanceOnly))
                         st_vec(p.x + (uint64_t)i * p.lds + t0 + off, xn[pass]);
                     if ((flags & kItemLast) && p.any_exchange) {

@@ -30,7 +30,9 @@ class RunConfig:
     asynchronous: bool = False      # workers reach the master one at a time, seeded order
     sync_free: str = "no"           # "yes": weights on the device (easgd_exchange_dynamic);
                                     # "mixed": device and host forms of the rule alternate
-    fused: str = "no"               # exchange rounds in one pass: "given" (coefficients known
+    fused: str = "no"               # "next": the exchange rides on the next round's local step
+                                    # (easgd_exchange_then_step; needs tau >= 2); or the
+                                    # exchange round in one pass: "given" (coefficients known
                                     # before the step: alpha) or "lagged" (the rule's output
                                     # of the previous exchange round, kept on the device)
     method: str = "adahessian"      # local step: "adahessian", "sgd" or "msgd" (momentum)
@@ -65,7 +67,7 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
     alpha = cfg.alpha_value()
     log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "orders_equal": True,
            "exchanges": 0}
-    lagged_weights = None
+    lagged_weights = pending = None
     for t in range(1, cfg.rounds + 1):
         mask_g = h.dw_mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
         mask_o = ref.mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
@@ -77,6 +79,50 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         common = dict(lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
                       hessian_power=cfg.hessian_power, weight_decay=cfg.weight_decay,
                       want_dist=ex)
+        if cfg.fused == "next":
+            # the library defers each exchange to the local step of the following round; the
+            # oracle exchanges at once.  States agree whenever no exchange is pending.
+            if pending is not None:
+                p_mask, p_order, p_h2, p_h1 = pending
+                h.easgd_exchange_then_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
+                                           active=mask_g if cfg.frozen else None, worker_mask=p_mask,
+                                           alpha=alpha, order=p_order, asynchronous=cfg.asynchronous,
+                                           dynamic=cfg.dynamic,
+                                           **{q: v for q, v in common.items() if q != "want_dist"})
+                if cfg.dynamic:
+                    w = h.ah_state_get(binding.AH_WEIGHTS)
+                    log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], p_h2) and
+                                                 np.array_equal(w[cfg.K:], p_h1))
+                pending = None
+                assert not ex, "tau >= 2"
+            else:
+                h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
+                                active=mask_g if cfg.frozen else None, **common)
+            ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
+                           active=mask_o if cfg.frozen else None, **common)
+            if ex:
+                log["exchanges"] += 1
+                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+                order_g = order_o = None
+                if cfg.asynchronous:
+                    order_g = h.dw_order_next(ORDER_SEED, t)
+                    order_o = ref.order_next(ORDER_SEED, t)
+                    log["orders_equal"] &= bool(np.array_equal(order_g, order_o))
+                h2, h1 = ref.weights_next(alpha) if cfg.dynamic else (None, None)
+                if cfg.asynchronous:
+                    ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
+                else:
+                    ref.exchange(mask_o, h2, h1, alpha=alpha)
+                pending = (mask_g, order_g, h2, h1)
+                if t == cfg.rounds:                                  # nothing follows: exchange now
+                    if cfg.dynamic:
+                        h.easgd_exchange_dynamic(mask_g, alpha, order_g, cfg.asynchronous)
+                    elif cfg.asynchronous:
+                        h.easgd_exchange_async(mask_g, None, alpha, order_g)
+                    else:
+                        h.easgd_exchange(mask_g, None, alpha)
+                    pending = None
+            continue
         if cfg.fused != "no" and ex:
             # one pass: step, distances, pull.  The oracle takes the same steps one by one.
             log["exchanges"] += 1

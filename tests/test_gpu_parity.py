@@ -406,6 +406,71 @@ def test_fused_rounds_with_lagged_dynamic_weights(B, torch, asyn, frozen):
     h.close()
 
 
+@pytest.mark.parametrize("asyn,frozen,dynamic", [(False, False, True), (True, False, True),
+                                                 (False, True, True), (True, False, False)])
+def test_exchange_riding_on_the_next_local_step(B, torch, asyn, frozen, dynamic):
+    # every exchange is deferred to the next round's local step (one pass instead of two);
+    # same coefficients, same bits as exchanging at once
+    layout = W.resnet18_layout(8)
+    cfg = RunConfig(K=8, segments=W.segments(layout), P=W.total_params(layout), rounds=100, tau=2,
+                    p_fail=0.25, max_stale=4 if frozen else 1, frozen=frozen, dynamic=dynamic,
+                    alpha=0.1 if asyn else None, asynchronous=asyn, fused="next")
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"] and log["orders_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    assert log["exchanges"] == 50
+    h.close()
+
+
+@pytest.mark.parametrize("layout", ["odd", "one", "ragged"])
+def test_exchange_then_step_equals_the_two_calls(B, torch, layout):
+    K = 4
+    if layout == "odd":
+        segs, P = ODD_SEGS, ODD_P
+    elif layout == "one":
+        segs, P, K = [], 1, 1
+    else:
+        segs, P, K = [(0, 1026, 3)], 2051, 2
+    ld = W.padded_ld(P)
+    rng = np.random.default_rng(80 + P)
+    theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
+    x0 = theta0[None] + rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.05)
+    h = B.Handle(K, P, segs)
+    ref = OracleState(theta0, K, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x0)
+    ref.x[:] = x0
+    for t in range(1, 7):
+        g = np.zeros((K, ld), np.float32)
+        hv = np.zeros((K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        hv[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        active = None if t % 3 else (rng.random(K) > 0.4).astype(np.uint8)
+        mask = None if t % 4 == 1 else (rng.random(K) > 0.3).astype(np.uint8)
+        asyn = t % 2 == 0
+        order = h.dw_order_next(6, t) if asyn else None
+        h2 = rng.uniform(0, 0.15, K).astype(np.float32)
+        h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+        h.easgd_exchange_then_step(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda(), Z_SEED, lr=0.01,
+                                   round_=t, active=active, worker_mask=mask,
+                                   weights=np.concatenate([h2, h1]), order=order, asynchronous=asyn)
+        if asyn:
+            ref.exchange_async(mask, h2, h1, order=order)
+        else:
+            ref.exchange(mask, h2, h1)
+        ref.local_step(g, hv, Z_SEED, t, lr=0.01, active=active)
+        for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v), (B.AH_CENTER, ref.center)):
+            assert np.array_equal(h.ah_state_get(which), want), (t, which)
+    g = torch.zeros(K, ld, device="cuda")
+    with pytest.raises(B.AdaHessError) as e:                   # no distances pending for the rule
+        h.easgd_exchange_then_step(g, g, 1, lr=0.1, alpha=0.1, dynamic=True)
+    assert e.value.status == B.AH_ERR_STATE
+    h.close()
+
+
 def test_fused_round_argument_checks(B, torch):
     K, P = 2, 1000
     h = B.Handle(K, P, [])
@@ -646,7 +711,8 @@ def _full_size_run(B, kind, K, tau, rounds, p_fail, max_stale=1, frozen=False, n
     _check_run(B, cfg, _layout_inputs(layout, K, n_pool=n_pool))
 
 
-@pytest.mark.parametrize("variant", ["async_device_weights", "fused_lagged", "fused_lagged_async", "eamsgd"])
+@pytest.mark.parametrize("variant", ["async_device_weights", "fused_lagged", "fused_lagged_async", "eamsgd",
+                                     "exchange_with_next_step"])
 def test_full_size_resnet18_layout_variants(B, torch, variant):
     # config 2 at its full size with the other forms of the round, in the launch shapes the
     # bench times: two communication periods each, every element compared with the oracle
@@ -658,6 +724,8 @@ def test_full_size_resnet18_layout_variants(B, torch, variant):
         cfg = RunConfig(fused="lagged", **kw)
     elif variant == "fused_lagged_async":
         cfg = RunConfig(fused="lagged", asynchronous=True, alpha=0.1, **kw)
+    elif variant == "exchange_with_next_step":
+        cfg = RunConfig(fused="next", **kw)
     else:
         cfg = RunConfig(method="msgd", dynamic=False, alpha=0.1, asynchronous=True, **kw)
     h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, 8, n_pool=2), variant="omp")
