@@ -267,7 +267,7 @@ def gpu_arm(args):
     asyn = args.exchange == "async"
     # with a period of one round every step also measures distances, which cannot ride along
     ride = (args.exchange_pass == "next-step" and args.method == "adahessian" and not args.fused
-            and tau >= 2)
+            and tau >= 2 and args.samples == 1)      # the one-pass forms take one Hutchinson sample
     carry = {} if ride else None
     for _ in range(args.warmup):
         t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused,
