@@ -153,6 +153,23 @@ LAYOUTS = {
 }
 
 
+def random_segment_table(seed: int, target: int = 12_000, max_block: int = 128):
+    """A seeded, irregular tensor table for edge-case tests: (segments, P) with tensors of
+    every size from one block to a few thousand elements, spatial blocks from 1 to
+    max_block (3 x 3 kernels most often), occasional gaps, and a ragged end."""
+    rng = np.random.default_rng(seed)
+    segs, pos = [], int(rng.integers(0, 6))
+    while pos < target:
+        if rng.random() < 0.2:
+            pos += int(rng.integers(1, 40))                        # a gap: behaves as block 1
+        kind = rng.random()
+        block = 9 if kind < 0.4 else 1 if kind < 0.65 else int(rng.integers(2, max_block + 1))
+        length = block * int(rng.integers(1, max(2, min(400, 3000 // block))))
+        segs.append((pos, length, block))
+        pos += length
+    return segs, pos + int(rng.integers(0, 7))
+
+
 def total_params(layout) -> int:
     return layout[-1].offset + layout[-1].numel if layout else 0
 

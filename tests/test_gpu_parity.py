@@ -84,6 +84,41 @@ def test_local_step_matches_oracle(B, torch, segs, P, hp, wd):
     h.close()
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_local_step_random_segment_tables(B, torch, seed):
+    # irregular tensor tables: every block size up to 128, blocks across tile edges, many
+    # tensors inside one tile, gaps, odd offsets, ragged ends; plain, distance, n-sample and
+    # one-pass forms of the step
+    segs, P = W.random_segment_table(100 + seed)
+    K, ld = 3, W.padded_ld(P)
+    rng = np.random.default_rng(seed)
+    theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
+    h = B.Handle(K, P, segs)
+    ref = OracleState(theta0, K, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    for t in range(1, 7):
+        n = 2 if t == 3 else 1
+        g = np.zeros((K, ld), np.float32)
+        hv = np.zeros((n, K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.1)
+        hv[:, :, :P] = rng.standard_normal((n, K, P)).astype(np.float32) * np.float32(0.1)
+        gd = torch.from_numpy(g).cuda()
+        hd = torch.from_numpy(hv if n > 1 else hv[0]).cuda()
+        if t == 5:      # exchange, then this step, in one pass
+            h.easgd_exchange_then_step(gd, hd, Z_SEED, lr=0.01, round_=t, alpha=0.2)
+            ref.exchange(alpha=0.2)
+            ref.local_step(g, hv[0], Z_SEED, t, lr=0.01)
+        else:
+            h.ah_local_step(gd, hd, Z_SEED, lr=0.01, round_=t, want_dist=t % 2 == 0)
+            ref.local_step(g, hv if n > 1 else hv[0], Z_SEED, t, lr=0.01, want_dist=t % 2 == 0)
+        if t % 2 == 0:
+            assert np.array_equal(h.ah_state_get(B.AH_NORM2), ref.norm2), t
+    for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v), (B.AH_CENTER, ref.center)):
+        assert np.array_equal(h.ah_state_get(which), want), which
+    h.close()
+
+
 def test_local_step_inactive_padding_and_auto_round(B, torch):
     segs, P, K = ODD_SEGS, ODD_P, 4
     theta0, pool = _inputs(segs, P, K, 1, seed=5)

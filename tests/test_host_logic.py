@@ -128,9 +128,11 @@ def test_weights_match_oracle_bit_for_bit_given_same_distances(B):
         h.close()
 
 
-@pytest.mark.parametrize("name", ["resnet18", "resnet50", "vgg16", "odd"])
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "vgg16", "odd"] + [f"random{k}" for k in range(12)])
 def test_tile_descriptors_cover_whole_blocks(B, name):
-    if name == "odd":
+    if name.startswith("random"):
+        segs, P = W.random_segment_table(int(name[6:]))
+    elif name == "odd":
         segs = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 128)]
         P = 13_111
     else:
