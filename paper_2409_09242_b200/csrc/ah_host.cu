@@ -405,6 +405,8 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     h->calls += 1;
     p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
     p.nrows = 0;
+    uint16_t idle[AH_MAX_WORKERS];
+    uint32_t nidle = 0;
     for (int q = 0; q < h->K; ++q) {
         // a fused round walks the workers in their arrival order
         const int i = fx && fx->asynchronous && fx->order ? (int)fx->order[q] : q;
@@ -416,7 +418,10 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         p.h2w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[i] : fx->alpha) : 0.f;
         p.h1w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[h->K + i] : fx->alpha) : 0.f;
         if (on) h->step[i] += 1;
-        if (on || dist || meets) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
+        // distances cover every worker; in a plain distance round the workers that sit
+        // the step out are measured by a streaming kernel of their own
+        if (on || meets || (dist && fx)) p.row[p.nrows++] = (uint16_t)i;
+        else if (dist) idle[nidle++] = (uint16_t)i;
         // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
         // (a worker that sat out steps has taken fewer); double, then one rounding
         const double t = (double)(h->step[i] ? h->step[i] : 1u);
@@ -429,6 +434,10 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     p.nitems = fx ? (p.nrows ? h->ntiles : 0u) : p.nrows * h->ntiles;
     AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
     if (p.nitems) h->launches += 1;
+    if (nidle) {
+        AH_CUDA(h, launch_distance_rows(h, idle, nidle));
+        h->launches += 1;
+    }
     if (dist) {
         const int rc = finish_distances(h);
         if (rc != AH_OK) return rc;
