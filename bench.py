@@ -188,7 +188,13 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
             e0.record()
         first_order = method != "adahessian"     # EASGD / EAMSGD: fixed alpha, no distances
         rode = False
-        if first_order:
+        if first_order and carry is not None and carry.get("pending") is not None:
+            rode = True
+            p_mask, p_order = carry.pop("pending")
+            h.easgd_exchange_then_sgd_step(g, SGD_LR, SGD_MOMENTUM if method == "msgd" else 0.0,
+                                           active=mask if frozen else None, worker_mask=p_mask,
+                                           alpha=alpha, order=p_order, asynchronous=asynchronous)
+        elif first_order:
             h.sgd_local_step(g, SGD_LR, SGD_MOMENTUM if method == "msgd" else 0.0,
                              active=mask if frozen else None)
         elif carry is not None and carry.get("pending") is not None:
@@ -211,7 +217,7 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         if events is not None:
             e1.record()
             events.append((e0, e1, 2 if rode else int(ex), n_act))
-        if ex and carry is not None and not first_order:
+        if ex and carry is not None:
             carry["pending"] = (mask, h.dw_order_next(ORDER_SEED, t) if asynchronous else None)
             exchanged += int(mask.sum())
         elif ex and fused and not first_order:
@@ -280,8 +286,10 @@ def gpu_arm(args):
     t = 0
     asyn = args.exchange == "async"
     # with a period of one round every step also measures distances, which cannot ride along
-    ride = (args.exchange_pass == "next-step" and args.method == "adahessian" and not args.fused
-            and tau >= 2 and args.samples == 1)      # the one-pass forms take one Hutchinson sample
+    # (with several Hutchinson samples the one-pass form fits fewer CTAs per SM and was
+    # measured slower than the separate exchange kernel)
+    ride = (args.exchange_pass == "next-step" and not args.fused and tau >= 2
+            and (args.samples == 1 or args.method != "adahessian"))
     carry = {} if ride else None
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -316,7 +324,11 @@ def gpu_arm(args):
         # the last timed period's exchange would ride on the next step; the first timed
         # period carried the one before it.  Launch it now, outside the timed region.
         p_mask, p_order = carry.pop("pending")
-        h.easgd_exchange_dynamic(p_mask, alpha_for(K), p_order, asyn)
+        if args.method != "adahessian":
+            (h.easgd_exchange_async(p_mask, None, alpha_for(K), p_order) if asyn
+             else h.easgd_exchange(p_mask, None, alpha_for(K)))
+        else:
+            h.easgd_exchange_dynamic(p_mask, alpha_for(K), p_order, asyn)
     wall1 = time.time()
     clocks = None
     if rank == 0:
@@ -368,7 +380,7 @@ def gpu_arm(args):
                 "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None,
                 "exchange_plus_step_ms": round(sum(rides) / len(rides), 4) if rides else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
-    if (args.fused or ride) and args.method == "adahessian":
+    if (args.fused and args.method == "adahessian") or ride:
         # fused exchange rounds: x crosses HBM once; the master row is read and written once
         run_bytes = bpu * P * worker_steps + 8 * P * args.steps
     else:

@@ -236,7 +236,7 @@ int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *h
  *       alpha while the rule has not yet run there.  This is the
  *       paper's "estimate of the master model": the score follows the distances with a
  *       delay of one communication period, and no call waits for the GPU.
- * One Hutchinson sample per step.  Memory traffic: 32 bytes per parameter update plus 8
+ * Memory traffic: 32 bytes per parameter update (one Hutchinson sample) plus 8
  * per parameter for the master row, 8 per (worker, parameter) less than the two calls.
  * Errors: INVALID_ARG, ALIGN, STATE, CUDA. */
 int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
@@ -256,13 +256,24 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
  *       STATE if no distances are pending), and the pass reads its output.
  * worker_mask says who takes part in the exchange; hy->active who takes the step.
  * hy->want_dist must be 0 (the distances to the new master are only defined once every
- * worker has met it) and hy->n_samples at most 1: with a communication period of one
- * round use ah_local_step_exchange or the separate calls.  Nothing waits for the GPU.
+ * worker has met it): with a communication period of one round use
+ * ah_local_step_exchange or the separate calls.  Nothing waits for the GPU.
  * Errors: INVALID_ARG, ALIGN, STATE, CUDA. */
 int easgd_exchange_then_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
                              uint64_t z_seed, const ah_hyper *hy, const uint8_t *worker_mask,
                              const float *weights, float alpha, const uint16_t *order,
                              int asynchronous, int dynamic);
+
+/* The first-order counterpart of easgd_exchange_then_step: the exchange of the round
+ * just finished (easgd_exchange, or easgd_exchange_async with `order` when
+ * asynchronous != 0; weights host 2K floats or NULL = alpha for all, the fixed moving
+ * rate of EASGD / EAMSGD) and the next sgd_local_step in one pass over x; bit for bit
+ * the two calls in sequence.  hy->want_dist must be 0.  Traffic: 12 bytes per update
+ * (20 with momentum) + 8 per parameter, instead of + 8 per (worker, parameter) + 8.
+ * Errors: INVALID_ARG, ALIGN, STATE, CUDA. */
+int easgd_exchange_then_sgd_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *hy,
+                                 const uint8_t *worker_mask, const float *weights, float alpha,
+                                 const uint16_t *order, int asynchronous);
 
 /* Parameters of the dynamic weighting rule (Sec. V-B): history depth p, the
  * coefficients c_0..c_{p-1} of Eqs. 10-11 (c_0 weighs the newest difference; they

@@ -36,7 +36,7 @@ EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_st
            "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step",
            "ah_local_step_exchange", "easgd_exchange_then_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "dw_partition", "ah_distances_static", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "easgd_exchange_then_sgd_step", "dw_partition", "ah_distances_static", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -84,6 +84,9 @@ _lib.dw_mask_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.c_double, C.c_int,
                               C.POINTER(C.c_uint8)]
 _lib.easgd_exchange.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float]
 _lib.sgd_local_step.argtypes = [_vp, _vp, C.c_uint64, C.POINTER(sgd_hyper)]
+_lib.easgd_exchange_then_sgd_step.argtypes = [_vp, _vp, C.c_uint64, C.POINTER(sgd_hyper),
+                                              C.POINTER(C.c_uint8), C.POINTER(C.c_float), C.c_float,
+                                              C.POINTER(C.c_uint16), C.c_int]
 _lib.dw_partition.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, C.POINTER(C.c_uint32),
                               C.POINTER(C.c_uint64)]
 _lib.dw_order_next.argtypes = [_vp, C.c_uint64, C.c_uint32, C.POINTER(C.c_uint16)]
@@ -177,6 +180,17 @@ def _dev_ptr(t, name):
     if t.dim() == 2 and t.stride(1) != 1:
         raise ValueError(f"{name}: rows must be contiguous")
     return t.data_ptr()
+
+
+def _hvp_samples(grad, hvp):
+    """(n_samples, sample stride) of hvp given as [K, ld] or as [n, K, ld]."""
+    if hvp.dim() == 3:
+        if hvp.stride(2) != 1 or hvp.shape[1:] != grad.shape or hvp.stride(1) != grad.stride(0):
+            raise ValueError("hvp: [n, K, ld] with the shape and row stride of grad")
+        return int(hvp.shape[0]), int(hvp.stride(0))
+    if grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
+        raise ValueError("grad and hvp must share shape and row stride")
+    return 1, 0
 
 
 class Handle:
@@ -302,13 +316,7 @@ class Handle:
                       hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
                       want_dist=False):
         """hvp: [K, ld] for one Hutchinson sample, or [n, K, ld] for n samples per step."""
-        n_samples, sample_stride = 1, 0
-        if hvp.dim() == 3:
-            n_samples, sample_stride = hvp.shape[0], hvp.stride(0)
-            if hvp.stride(2) != 1 or hvp.shape[1:] != grad.shape or hvp.stride(1) != grad.stride(0):
-                raise ValueError("hvp: [n, K, ld] with the shape and row stride of grad")
-        elif grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
-            raise ValueError("grad and hvp must share shape and row stride")
+        n_samples, sample_stride = _hvp_samples(grad, hvp)
         act = None
         if active is not None:
             act = np.ascontiguousarray(active, np.uint8)
@@ -336,8 +344,7 @@ class Handle:
                                hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
                                want_dist=False, worker_mask=None, weights=None, alpha=0.0, order=None,
                                asynchronous=False, lagged=False):
-        if grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
-            raise ValueError("grad and hvp must share shape and row stride")
+        n_samples, sample_stride = _hvp_samples(grad, hvp)
         act = m = w = o = None
         if active is not None:
             act = np.ascontiguousarray(active, np.uint8)
@@ -358,9 +365,9 @@ class Handle:
             o = order.ctypes.data_as(C.POINTER(C.c_uint16))
         hy = ah_hyper(lr, beta1, beta2, eps, hessian_power, weight_decay, int(round_),
                       act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None,
-                      1 if want_dist else 0, 1, 0)
+                      1 if want_dist else 0, n_samples, sample_stride)
         self._check(_lib.ah_local_step_exchange(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
-                                                grad.stride(0), int(z_seed), C.byref(hy), m, w, alpha, o,
+                                                grad.stride(-2), int(z_seed), C.byref(hy), m, w, alpha, o,
                                                 1 if asynchronous else 0, 1 if lagged else 0),
                     "ah_local_step_exchange")
 
@@ -368,8 +375,7 @@ class Handle:
                                  hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
                                  worker_mask=None, weights=None, alpha=0.0, order=None,
                                  asynchronous=False, dynamic=False):
-        if grad.shape != hvp.shape or grad.stride(0) != hvp.stride(0):
-            raise ValueError("grad and hvp must share shape and row stride")
+        n_samples, sample_stride = _hvp_samples(grad, hvp)
         act = m = w = o = None
         if active is not None:
             act = np.ascontiguousarray(active, np.uint8)
@@ -389,11 +395,39 @@ class Handle:
                 raise ValueError("order: K entries")
             o = order.ctypes.data_as(C.POINTER(C.c_uint16))
         hy = ah_hyper(lr, beta1, beta2, eps, hessian_power, weight_decay, int(round_),
-                      act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None, 0, 1, 0)
+                      act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None, 0,
+                      n_samples, sample_stride)
         self._check(_lib.easgd_exchange_then_step(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
-                                                  grad.stride(0), int(z_seed), C.byref(hy), m, w, alpha,
+                                                  grad.stride(-2), int(z_seed), C.byref(hy), m, w, alpha,
                                                   o, 1 if asynchronous else 0, 1 if dynamic else 0),
                     "easgd_exchange_then_step")
+
+    def easgd_exchange_then_sgd_step(self, grad, lr, momentum=0.0, active=None, worker_mask=None,
+                                     weights=None, alpha=0.0, order=None, asynchronous=False):
+        act = m = w = o = None
+        if active is not None:
+            act = np.ascontiguousarray(active, np.uint8)
+            if act.size != self.K:
+                raise ValueError("active: K bytes")
+        if worker_mask is not None:
+            worker_mask = np.ascontiguousarray(worker_mask, np.uint8)
+            m = worker_mask.ctypes.data_as(C.POINTER(C.c_uint8))
+        if weights is not None:
+            weights = np.ascontiguousarray(weights, np.float32)
+            if weights.size != 2 * self.K:
+                raise ValueError("weights: 2K floats (h2 then h1)")
+            w = weights.ctypes.data_as(C.POINTER(C.c_float))
+        if order is not None:
+            order = np.ascontiguousarray(order, np.uint16)
+            if order.size != self.K:
+                raise ValueError("order: K entries")
+            o = order.ctypes.data_as(C.POINTER(C.c_uint16))
+        hy = sgd_hyper(lr, momentum,
+                       act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None, 0)
+        self._check(_lib.easgd_exchange_then_sgd_step(self._h, _dev_ptr(grad, "grad"), grad.stride(0),
+                                                      C.byref(hy), m, w, alpha, o,
+                                                      1 if asynchronous else 0),
+                    "easgd_exchange_then_sgd_step")
 
     def dw_config(self, p_hist, c, kappa):
         c = np.ascontiguousarray(c, np.float64)

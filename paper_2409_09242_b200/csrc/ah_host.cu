@@ -463,7 +463,6 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
                            int asynchronous, int lagged)
 {
     if (!hy) return AH_ERR_INVALID_ARG;
-    if (hy->n_samples > 1) return AH_ERR_INVALID_ARG;          // one Hutchinson sample when fused
     if (lagged && (!hy->want_dist || weights)) return AH_ERR_INVALID_ARG;
     FusedExchange fx;
     fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;
@@ -478,7 +477,7 @@ int easgd_exchange_then_step(ah_ctx *h, const float *grad, const float *hvp, uin
                              int asynchronous, int dynamic)
 {
     if (!hy) return AH_ERR_INVALID_ARG;
-    if (hy->n_samples > 1 || hy->want_dist) return AH_ERR_INVALID_ARG;
+    if (hy->want_dist) return AH_ERR_INVALID_ARG;
     if (dynamic && weights) return AH_ERR_INVALID_ARG;
     FusedExchange fx;
     fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;

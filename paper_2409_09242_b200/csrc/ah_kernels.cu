@@ -833,7 +833,10 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
 template <int POWMODE, bool WD>
 static cudaError_t launch_step_dist(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
 {
-    if (p.fused)                         // step and exchange in one pass (one Hutchinson sample)
+    if (p.fused && p.nsamp > 1u)         // step and exchange in one pass, several samples
+        return want_dist ? launch_step_one<POWMODE, WD, true, true, true>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, true, true>(p, sm_count, s);
+    if (p.fused)                         // step and exchange in one pass
         return want_dist ? launch_step_one<POWMODE, WD, true, false, true>(p, sm_count, s)
                          : launch_step_one<POWMODE, WD, false, false, true>(p, sm_count, s);
     if (p.nsamp > 1u)

@@ -103,6 +103,102 @@ static cudaError_t launch_sgd(const SgdParams &p, cudaStream_t s)
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// Exchange, then the first-order step, in one pass (EASGD / EAMSGD periods): one thread
+// owns four consecutive columns, keeps their master values in registers and walks the
+// workers in arrival order; each worker's x is pulled (Eqs. 12-13), stepped, and stored
+// once.  Loads of the next workers are in flight while one is computed.
+// ---------------------------------------------------------------------------
+struct SgdExchangeParams {
+    float *x, *u, *c;
+    const float *grad;
+    const float *wdev;             // not null: h2 of worker i at wdev[i], h1 at wdev[K + i]
+    uint64_t lds, ld;
+    uint32_t nvec;                 // float4 columns (= lds / 4)
+    uint32_t P;
+    float lr, momentum;
+    uint32_t nrows, nworkers, asynchronous, any_exchange;
+    uint16_t row[AH_MAX_WORKERS];  // workers in arrival order
+    uint8_t active[AH_MAX_WORKERS], exch[AH_MAX_WORKERS];   // by worker index
+    float h1w[AH_MAX_WORKERS], h2w[AH_MAX_WORKERS];
+};
+
+template <bool MOMENTUM>
+__global__ void __launch_bounds__(256)
+exchange_then_sgd_kernel(const __grid_constant__ SgdExchangeParams p)
+{
+    constexpr int kDepth = 2;                      // workers whose loads are in flight
+    const uint32_t q = blockIdx.x * 256u + threadIdx.x;
+    if (q >= p.nvec) return;
+    const uint64_t col = 4ull * q;
+    const int nv = p.P - (uint32_t)col >= 4u ? 4 : (int)(p.P - (uint32_t)col);   // lanes past P stay zero
+    const float4 c_old = ld_vec(p.c + col);
+    float4 carry = p.asynchronous ? c_old : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (uint32_t r0 = 0; r0 < p.nrows; r0 += kDepth) {
+        float4 x[kDepth], g[kDepth], u[kDepth];
+#pragma unroll
+        for (int k = 0; k < kDepth; ++k) {
+            if (r0 + k < p.nrows) {
+                const uint32_t i = p.row[r0 + k];
+                x[k] = ld_vec(p.x + (uint64_t)i * p.lds + col);
+                if (p.active[i]) {
+                    g[k] = ld_vec(p.grad + (uint64_t)i * p.ld + col);
+                    if (MOMENTUM) u[k] = ld_vec(p.u + (uint64_t)i * p.lds + col);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kDepth; ++k) {
+            if (r0 + k < p.nrows) {
+                const uint32_t i = p.row[r0 + k];
+                if (p.exch[i]) {
+                    const float h1 = p.wdev ? p.wdev[p.nworkers + i] : p.h1w[i];
+                    const float h2 = p.wdev ? p.wdev[i] : p.h2w[i];
+                    float *xe = &x[k].x, *ae = &carry.x;
+                    const float *ce = &c_old.x;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (p.asynchronous) {
+                            const float d = __fsub_rn(xe[e], ae[e]);
+                            xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+                            ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+                        } else {
+                            const float d = __fsub_rn(xe[e], ce[e]);
+                            ae[e] = __fadd_rn(ae[e], __fmul_rn(h2, d));
+                            xe[e] = __fsub_rn(xe[e], __fmul_rn(h1, d));
+                        }
+                    }
+                }
+                if (p.active[i]) {
+                    float *xe = &x[k].x, *ue = &u[k].x;
+                    const float *ge = &g[k].x;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (e < nv) {
+                            if (MOMENTUM) {
+                                ue[e] = __fsub_rn(__fmul_rn(p.momentum, ue[e]), __fmul_rn(p.lr, ge[e]));
+                                xe[e] = __fadd_rn(xe[e], ue[e]);
+                            } else {
+                                xe[e] = __fsub_rn(xe[e], __fmul_rn(p.lr, ge[e]));
+                            }
+                        }
+                    }
+                    if (MOMENTUM) st_vec(p.u + (uint64_t)i * p.lds + col, u[k]);
+                }
+                st_vec(p.x + (uint64_t)i * p.lds + col, x[k]);
+            }
+        }
+    }
+    if (p.any_exchange) {
+        float4 cn = carry;
+        if (!p.asynchronous) {
+            cn.x = __fadd_rn(c_old.x, cn.x); cn.y = __fadd_rn(c_old.y, cn.y);
+            cn.z = __fadd_rn(c_old.z, cn.z); cn.w = __fadd_rn(c_old.w, cn.w);
+        }
+        st_vec(p.c + col, cn);
+    }
+}
+
 }  // namespace ah
 
 // Tile partials of ||x_i - c||^2 for workers that take no step this round (their x is
@@ -154,5 +250,53 @@ extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const s
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
     if (p.nrows) h->launches += 1;
     if (dist) return finish_distances(h);
+    return AH_OK;
+}
+
+extern "C" int easgd_exchange_then_sgd_step(ah_ctx *h, const float *grad, uint64_t ld,
+                                            const sgd_hyper *hy, const uint8_t *worker_mask,
+                                            const float *weights, float alpha, const uint16_t *order,
+                                            int asynchronous)
+{
+    if (!h || !grad || !hy || ld < h->P) return AH_ERR_INVALID_ARG;
+    if (!h->has_device) return AH_ERR_STATE;
+    if (!(hy->momentum >= 0.f && hy->momentum < 1.f) || hy->want_dist) return AH_ERR_INVALID_ARG;
+    if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0) return AH_ERR_ALIGN;
+    if (order) {                                  // must name every worker exactly once
+        bool seen[AH_MAX_WORKERS] = {};
+        for (int q = 0; q < h->K; ++q) {
+            if (order[q] >= h->K || seen[order[q]]) return AH_ERR_INVALID_ARG;
+            seen[order[q]] = true;
+        }
+    }
+    SgdExchangeParams p;
+    p.x = h->x; p.u = h->m; p.c = h->c; p.grad = grad; p.wdev = nullptr;
+    p.lds = h->lds; p.ld = ld;
+    p.nvec = (uint32_t)(h->lds / 4); p.P = h->P;
+    p.lr = hy->lr; p.momentum = hy->momentum;
+    p.nworkers = (uint32_t)h->K;
+    p.asynchronous = asynchronous ? 1u : 0u;
+    p.any_exchange = 0u;
+    p.nrows = 0;
+    for (int q = 0; q < h->K; ++q) {
+        const int i = asynchronous && order ? (int)order[q] : q;
+        const bool on = !hy->active || hy->active[i] != 0;
+        const bool meets = !worker_mask || worker_mask[i] != 0;
+        p.active[i] = on ? 1 : 0;
+        p.exch[i] = meets ? 1 : 0;
+        if (meets) p.any_exchange = 1u;
+        p.h2w[i] = weights ? weights[i] : alpha;
+        p.h1w[i] = weights ? weights[h->K + i] : alpha;
+        if (on) h->step[i] += 1;
+        if (on || meets) p.row[p.nrows++] = (uint16_t)i;
+    }
+    h->calls += 1;
+    if (p.nrows == 0) return AH_OK;
+    const unsigned blocks = (p.nvec + 255u) / 256u;
+    if (hy->momentum != 0.f) exchange_then_sgd_kernel<true><<<blocks, 256, 0, h->stream>>>(p);
+    else                     exchange_then_sgd_kernel<false><<<blocks, 256, 0, h->stream>>>(p);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->launches += 1;
     return AH_OK;
 }

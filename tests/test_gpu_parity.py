@@ -407,6 +407,8 @@ def test_fused_round_equals_step_then_exchange(B, torch, layout, asyn):
             weights = np.concatenate([h2, h1])
         else:
             h2 = h1 = weights = None
+        if t in (4, 7):                                          # two Hutchinson samples
+            hv = np.stack([hv, np.roll(hv, 1, axis=0)])
         h.ah_local_step_exchange(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda(), Z_SEED, lr=0.01,
                                  round_=t, active=active, want_dist=dist, worker_mask=mask,
                                  weights=weights, alpha=0.1, order=order, asynchronous=asyn)
@@ -489,6 +491,8 @@ def test_exchange_then_step_equals_the_two_calls(B, torch, layout):
         order = h.dw_order_next(6, t) if asyn else None
         h2 = rng.uniform(0, 0.15, K).astype(np.float32)
         h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+        if t == 4:                                               # three Hutchinson samples
+            hv = np.stack([hv, hv[::-1].copy(), -hv])
         h.easgd_exchange_then_step(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda(), Z_SEED, lr=0.01,
                                    round_=t, active=active, worker_mask=mask,
                                    weights=np.concatenate([h2, h1]), order=order, asynchronous=asyn)
@@ -557,6 +561,49 @@ def test_easgd_eamsgd_rounds_reduced(B, torch, method, asyn):
     viol, bits = compare_state(h, ref, B)
     assert log["masks_equal"] and log["orders_equal"]
     assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    h.close()
+
+
+@pytest.mark.parametrize("K,P", [(1, 1), (2, 2051), (5, 13_111), (8, 184_837), (64, 3001)])
+@pytest.mark.parametrize("delta", [0.0, 0.5])
+def test_exchange_then_sgd_step_equals_the_two_calls(B, torch, K, P, delta):
+    # EASGD / EAMSGD periods in one pass per exchange: pull, then the first-order step
+    rng = np.random.default_rng(K * 11 + P)
+    ld = W.padded_ld(P) + 4
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    x0 = theta0[None] + rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.05)
+    h = B.Handle(K, P, [])
+    ref = OracleState(theta0, K, [])
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_state_set(B.AH_X, x0)
+    ref.x[:] = x0
+    for t in range(1, 8):
+        g = np.full((K, ld), np.nan, np.float32)             # columns past P must never be used
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32)
+        active = None if t % 3 else (rng.random(K) > 0.4).astype(np.uint8)
+        mask = None if t % 4 == 1 else (rng.random(K) > 0.3).astype(np.uint8)
+        if t == 6:
+            mask = np.zeros(K, np.uint8)
+        asyn = t % 2 == 0
+        order = h.dw_order_next(8, t) if asyn else None
+        if t % 3 == 1:
+            h2 = rng.uniform(0, 0.1, K).astype(np.float32)
+            h1 = rng.uniform(0.05, 1, K).astype(np.float32)
+            weights = np.concatenate([h2, h1])
+        else:
+            h2 = h1 = weights = None
+        h.easgd_exchange_then_sgd_step(torch.from_numpy(g).cuda(), 0.01, delta, active=active,
+                                       worker_mask=mask, weights=weights, alpha=0.1, order=order,
+                                       asynchronous=asyn)
+        if asyn:
+            ref.exchange_async(mask, h2, h1, alpha=0.1, order=order)
+        else:
+            ref.exchange(mask, h2, h1, alpha=0.1)
+        ref.sgd_step(g, 0.01, delta, active=active)
+        for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_CENTER, ref.center)):
+            assert np.array_equal(h.ah_state_get(which), want), (t, which)
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), ref.step)
+    assert not h.ah_state_get(B.AH_V).any()
     h.close()
 
 
