@@ -144,6 +144,46 @@ class ClockSampler:
                 "window": window, "reasons": reasons}
 
 
+class InputStager:
+    """End-to-end leg: the inputs of every round come from pinned host memory.  Two device
+    buffers and a copy stream: while round t computes from one buffer, the inputs of round
+    t + 1 are copied into the other."""
+
+    def __init__(self, host_pool, like, with_hvp):
+        import torch
+        self.host_pool, self.with_hvp = host_pool, with_hvp
+        self.bufs = [(torch.empty_like(like[0]), torch.empty_like(like[1])) for _ in range(2)]
+        self.copy_stream = torch.cuda.Stream()
+        self.ready = [torch.cuda.Event() for _ in range(2)]      # copy into buffer b finished
+        self.done = [torch.cuda.Event() for _ in range(2)]       # compute from buffer b finished
+        self.issued_for = None                                   # round whose copy is in flight
+
+    def _issue(self, t):
+        import torch
+        b = t % 2
+        hg, hh = self.host_pool[t % len(self.host_pool)]
+        with torch.cuda.stream(self.copy_stream):
+            self.copy_stream.wait_event(self.done[b])            # the buffer's last reader is through
+            self.bufs[b][0].copy_(hg, non_blocking=True)
+            if self.with_hvp:
+                self.bufs[b][1].copy_(hh, non_blocking=True)
+            self.ready[b].record(self.copy_stream)
+
+    def inputs(self, t):
+        """Device inputs of round t (the compute stream waits for their copy), and the copy
+        of round t + 1 started behind them."""
+        import torch
+        if self.issued_for != t:
+            self._issue(t)
+        torch.cuda.current_stream().wait_event(self.ready[t % 2])
+        self._issue(t + 1)
+        self.issued_for = t + 1
+        return self.bufs[t % 2]
+
+    def release(self, t):
+        self.done[t % 2].record()                                # on the compute stream
+
+
 def max_over_ranks(ms, dist, device):
     """The slowest rank's time: what a multi-GPU number is quoted on."""
     if dist is None:
@@ -161,9 +201,9 @@ def whole_job_updates_per_second(updates_per_rank, world, ms):
 
 def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_events=None,
                method="adahessian", sync_free=False, fused=False, carry=None):
-    """One communication period starting after round t0.  With `stage` = (host_pool,
-    dev_grad, dev_hvp) the inputs of every round are first copied from pinned host
-    memory (the end-to-end leg).  With `carry` (a dict kept by the caller) the exchange
+    """One communication period starting after round t0.  With `stage` (an InputStager)
+    the inputs of every round are first copied from pinned host memory (the end-to-end
+    leg).  With `carry` (a dict kept by the caller) the exchange
     of a period is not launched at its end but rides on the first local step of the next
     period (one pass over x instead of two, same result).  Returns (next t0, worker-steps
     taken, workers that exchanged)."""
@@ -176,11 +216,7 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         mask = h.dw_mask_next(MASK_SEED, t, p_fail, max_stale)
         ex = r == tau - 1
         if stage is not None:
-            host_pool, g, hv = stage
-            hg, hh = host_pool[t % len(host_pool)]
-            g.copy_(hg, non_blocking=True)
-            if method == "adahessian":
-                hv.copy_(hh, non_blocking=True)
+            g, hv = stage.inputs(t)
         else:
             g, hv = pool[t % len(pool)]
         if events is not None:
@@ -212,6 +248,8 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
         else:
             h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
                             **HYPER)      # hv is [K, ld], or [n, K, ld] with --samples n
+        if stage is not None:
+            stage.release(t)
         n_act = int(mask.sum()) if frozen else K
         worker_steps += n_act
         if events is not None:
@@ -404,15 +442,15 @@ def gpu_arm(args):
     if not args.no_e2e:
         n_host = 1 if pair_bytes > 4e9 else 2
         host_pool = [(g.cpu().pin_memory(), hv.cpu().pin_memory()) for g, hv in pool[:n_host]]
-        sg, sh = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
+        stager = InputStager(host_pool, pool[0], args.method == "adahessian")
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
-        t, _, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn,
+        t, _, _ = run_period(h, pool, t, wl, stage=stager, asynchronous=asyn,
                              method=args.method)      # the end-to-end leg reads the weights back
         barrier()
         start.record()
         e2e_ws = 0
         for _ in range(e2e_steps):
-            t, ws, _ = run_period(h, pool, t, wl, stage=(host_pool, sg, sh), asynchronous=asyn,
+            t, ws, _ = run_period(h, pool, t, wl, stage=stager, asynchronous=asyn,
                                   method=args.method)
             e2e_ws += ws
         stop.record()
