@@ -136,8 +136,9 @@ enum {
                           widened to whole spatial blocks [e0, e1); flags bit 0 = the tile
                           touches a block > 1, bit 1 = every such block is a 3 x 3 kernel
                           (get only, host)                                                  */
-    AH_WEIGHTS = 12    /* float  [2K]  h2[0..K) then h1[0..K) of the last
-                          easgd_exchange_dynamic (get only, host)                           */
+    AH_WEIGHTS = 12    /* float  [2K]  h2[0..K) then h1[0..K): the last output of the
+                          weighting rule on the device (host side only); part of a
+                          checkpoint when lagged one-pass rounds are used                   */
 };
 
 /* ---- life cycle ------------------------------------------------------------ */

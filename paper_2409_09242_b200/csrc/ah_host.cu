@@ -510,10 +510,16 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
         return AH_OK;
     }
     if (on_device) return AH_ERR_INVALID_ARG;
-    if (which == AH_WEIGHTS) {                 // coefficients of the last dynamic exchange
-        if (!to_user || !h->has_device) return to_user ? AH_ERR_STATE : AH_ERR_INVALID_ARG;
-        AH_CUDA(h, cudaMemcpyAsync(user, h->weights_dev, 2 * (size_t)h->K * sizeof(float),
-                                   cudaMemcpyDeviceToHost, h->stream));
+    if (which == AH_WEIGHTS) {                 // coefficients of the last rule run on the device
+        if (!h->has_device) return AH_ERR_STATE;
+        if (to_user) {
+            AH_CUDA(h, cudaMemcpyAsync(user, h->weights_dev, 2 * (size_t)h->K * sizeof(float),
+                                       cudaMemcpyDeviceToHost, h->stream));
+        } else {                               // restored from a checkpoint: a lagged round may use them
+            AH_CUDA(h, cudaMemcpyAsync(h->weights_dev, user, 2 * (size_t)h->K * sizeof(float),
+                                       cudaMemcpyHostToDevice, h->stream));
+            h->lagged_ready = true;
+        }
         AH_CUDA(h, cudaStreamSynchronize(h->stream));
         return AH_OK;
     }

@@ -754,6 +754,50 @@ def test_checkpoint_resume_is_bit_identical(B, torch):
     h_b.close()
 
 
+def test_checkpoint_resume_with_the_rule_on_the_device(B, torch):
+    # the same with lagged one-pass exchange rounds: the history ring lives on the device and
+    # the coefficients waiting for the next exchange round are part of the snapshot
+    layout = W.resnet18_layout(16)
+    segs, P, K, tau = W.segments(layout), W.total_params(layout), 4, 2
+    theta0, pool = _layout_inputs(layout, K)
+    dev_pool = [(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda()) for g, hv in pool]
+    from parity_driver import MASK_SEED
+
+    def rounds(h, first, last):
+        for t in range(first, last + 1):
+            mask = h.dw_mask_next(MASK_SEED, t, 0.2)
+            g, hv = dev_pool[t % len(dev_pool)]
+            if t % tau == 0:
+                h.ah_local_step_exchange(g, hv, Z_SEED, lr=0.01, round_=t, want_dist=True,
+                                         worker_mask=mask, alpha=0.05, lagged=True)
+            else:
+                h.ah_local_step(g, hv, Z_SEED, lr=0.01, round_=t)
+
+    def fresh():
+        h = B.Handle(K, P, segs)
+        h.ah_state_set(B.AH_CENTER, theta0)
+        h.ah_broadcast_center()
+        return h
+
+    h_full = fresh()
+    rounds(h_full, 1, 20)
+    h_a = fresh()
+    rounds(h_a, 1, 10)
+    snap = {w: h_a.ah_state_get(w) for w in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER, B.AH_STEP, B.AH_UHIST,
+                                             B.AH_DOWN_UNTIL, B.AH_ROUND, B.AH_WEIGHTS)}
+    h_a.close()
+    h_b = B.Handle(K, P, segs)
+    for w, val in snap.items():
+        h_b.ah_state_set(w, val)
+    rounds(h_b, 11, 20)
+    for w in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER, B.AH_WEIGHTS):
+        a, b = h_full.ah_state_get(w), h_b.ah_state_get(w)
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), w
+    assert np.array_equal(h_full.ah_state_get(B.AH_UHIST), h_b.ah_state_get(B.AH_UHIST))
+    h_full.close()
+    h_b.close()
+
+
 def test_error_paths_and_own_allocation(B, torch):
     K, P = 2, 1000
     h = B.Handle(K, P, [], own_alloc=True)           # cudaMalloc workspace, default stream
