@@ -523,6 +523,97 @@ def test_fused_round_argument_checks(B, torch):
     h.close()
 
 
+# ------------------------------------------- every form of the round, mixed at random
+@pytest.mark.parametrize("seed", range(6))
+def test_random_mix_of_round_forms(B, torch, seed):
+    """Each exchange round picks one of the seven ways the library offers to take it (host
+    or device rule, exchange kernel at once or riding on the next step, one pass with given
+    or lagged coefficients, simultaneous or asynchronous), plain rounds take one or two
+    Hutchinson samples; the oracle follows with its separate functions.  Checks that the
+    forms compose: history ring on host and device, pending distances, lagged weights."""
+    from parity_driver import MASK_SEED, ORDER_SEED
+    rng = np.random.default_rng(1000 + seed)
+    layout = W.resnet18_layout(16)
+    segs, P, K, tau, R, alpha = W.segments(layout), W.total_params(layout), 5, 3, 36, 0.08
+    ld = W.padded_ld(P)
+    theta0 = W.theta0_np(layout, seed)
+    h = B.Handle(K, P, segs)
+    ref = OracleState(theta0, K, segs)
+    h.ah_state_set(B.AH_CENTER, theta0)
+    h.ah_broadcast_center()
+    dev_w = None            # last output of the rule on the device (what a lagged round pulls with)
+    pending = None          # an exchange deferred to the next round's step
+    for t in range(1, R + 1):
+        ex = t % tau == 0
+        mask = h.dw_mask_next(MASK_SEED, t, 0.25)
+        assert np.array_equal(mask, ref.mask_next(MASK_SEED, t, 0.25))
+        n = 2 if rng.random() < 0.3 else 1
+        g = np.zeros((K, ld), np.float32)
+        hv = np.zeros((n, K, ld), np.float32)
+        g[:, :P] = rng.standard_normal((K, P)).astype(np.float32) * np.float32(0.05)
+        hv[:, :, :P] = rng.standard_normal((n, K, P)).astype(np.float32) * np.float32(0.05)
+        hv_o = hv if n > 1 else hv[0]
+        gd, hd = torch.from_numpy(g).cuda(), torch.from_numpy(hv_o).cuda()
+        asyn = bool(rng.random() < 0.5)
+        order = h.dw_order_next(ORDER_SEED, t) if asyn else None
+        if asyn:
+            assert np.array_equal(order, ref.order_next(ORDER_SEED, t))
+        form = rng.choice(["host", "device", "defer", "given", "lagged"]) if ex else None
+
+        def oracle_exchange(m, o, a, h2=None, h1=None):
+            if a:
+                ref.exchange_async(m, h2, h1, alpha=alpha, order=o)
+            else:
+                ref.exchange(m, h2, h1, alpha=alpha)
+
+        if pending is not None:                 # last round's exchange rides on this step
+            p_mask, p_order, p_asyn = pending
+            h.easgd_exchange_then_step(gd, hd, Z_SEED, lr=0.01, round_=t, worker_mask=p_mask, alpha=alpha,
+                                       order=p_order, asynchronous=p_asyn, dynamic=True)
+            dev_w = ref.weights_next(alpha)
+            w = h.ah_state_get(B.AH_WEIGHTS)
+            assert np.array_equal(w[:K], dev_w[0]) and np.array_equal(w[K:], dev_w[1]), t
+            oracle_exchange(p_mask, p_order, p_asyn, *dev_w)
+            ref.local_step(g, hv_o, Z_SEED, t, lr=0.01)
+            pending = None
+        elif form in ("given", "lagged"):       # this round's step and exchange in one pass
+            h.ah_local_step_exchange(gd, hd, Z_SEED, lr=0.01, round_=t, want_dist=True, worker_mask=mask,
+                                     alpha=alpha, order=order, asynchronous=asyn, lagged=form == "lagged")
+            ref.local_step(g, hv_o, Z_SEED, t, lr=0.01, want_dist=True)
+            if form == "lagged":
+                oracle_exchange(mask, order, asyn, *(dev_w if dev_w is not None else (None, None)))
+                dev_w = ref.weights_next(alpha)
+            else:
+                oracle_exchange(mask, order, asyn)
+            continue
+        else:
+            h.ah_local_step(gd, hd, Z_SEED, lr=0.01, round_=t, want_dist=ex)
+            ref.local_step(g, hv_o, Z_SEED, t, lr=0.01, want_dist=ex)
+        if form == "host":
+            w = h.dw_weights_next(alpha)
+            h2, h1 = ref.weights_next(alpha)
+            assert np.array_equal(w[:K], h2) and np.array_equal(w[K:], h1), t
+            if asyn:
+                h.easgd_exchange_async(mask, w, alpha, order)
+            else:
+                h.easgd_exchange(mask, w, alpha)
+            oracle_exchange(mask, order, asyn, h2, h1)
+        elif form == "device":
+            h.easgd_exchange_dynamic(mask, alpha, order, asyn)
+            dev_w = ref.weights_next(alpha)
+            oracle_exchange(mask, order, asyn, *dev_w)
+        elif form == "defer":
+            pending = (mask, order, asyn)
+    if pending is not None:
+        p_mask, p_order, p_asyn = pending
+        h.easgd_exchange_dynamic(p_mask, alpha, p_order, p_asyn)
+        oracle_exchange(p_mask, p_order, p_asyn, *ref.weights_next(alpha))
+    for which, want in ((B.AH_X, ref.x), (B.AH_M, ref.m), (B.AH_V, ref.v), (B.AH_CENTER, ref.center)):
+        assert np.array_equal(h.ah_state_get(which), want), which
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    h.close()
+
+
 # ------------------------------------------- first-order local steps (EASGD / EAMSGD)
 @pytest.mark.parametrize("K,P", [(1, 1), (2, 1023), (3, 4097), (4, 184_837), (8, 4 * 1024 * 5), (5, 8193)])
 @pytest.mark.parametrize("delta", [0.0, 0.5])
