@@ -3,7 +3,11 @@
 oracle, element by element.  Too long for the test suite (the oracle needs minutes per
 configuration): run by hand on a machine with a B200,
 
-    python tests/run_full_configs.py [c3 c4 c5 ...] > full_configs.txt
+    python tests/run_full_configs.py [--ride] [c3 c4 c5 ...] > full_configs.txt
+
+With --ride every exchange is deferred to the next round's local step
+(easgd_exchange_then_step, the launch shape the benchmark times by default; runs with a
+communication period of one round are skipped).
 
 It prints one line per run: violations of |gpu - oracle| <= 1e-6 + 1e-5 |oracle| and the
 number of elements whose bits differ, for x, m, v and the master, and whether masks,
@@ -44,8 +48,15 @@ def runs(which):
 def main():
     import torch
     torch.cuda.set_device(0)
-    which = sys.argv[1:] or ["c2", "c3", "c4", "c5"]
+    args = sys.argv[1:]
+    ride = "--ride" in args
+    which = [a for a in args if a != "--ride"] or ["c2", "c3", "c4", "c5"]
     for name, kind, kw in runs(which):
+        if ride:
+            if kw["tau"] < 2:
+                continue
+            kw = dict(kw, fused="next")
+            name += " (exchange riding on the next step)"
         layout = W.LAYOUTS[kind]()
         cfg = RunConfig(segments=W.segments(layout), P=W.total_params(layout), **kw)
         t0 = time.time()
