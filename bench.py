@@ -43,6 +43,11 @@ WORKLOADS = {
     "c5k16": ("resnet50", 16, 4, 0.1, 1, False),
     "c5k32": ("resnet50", 32, 4, 0.1, 1, False),
     "c5k64": ("resnet50", 64, 4, 0.1, 1, False),
+    # the paper's own setting (Sec. VI-VII): its small CNN, 4 or 8 workers, tau in {1, 2, 4},
+    # communication suppressed one third of the time
+    "paper_k4_tau4": ("mnist_cnn", 4, 4, 1 / 3, 1, False),
+    "paper_k8_tau2": ("mnist_cnn", 8, 2, 1 / 3, 1, False),
+    "paper_k8_tau1": ("mnist_cnn", 8, 1, 1 / 3, 1, False),
     # small cases for profiler captures (about 1 GB on the device, still far above L2)
     "p18k4": ("resnet18", 4, 4, 0.1, 1, False),
     "pvggk1": ("vgg16", 1, 4, 0.1, 1, False),

@@ -728,6 +728,18 @@ def _layout_inputs(layout, K, n_pool=3, seed=0):
     return W.theta0_np(layout, seed), W.gaussian_pool_np(layout, K, n_pool, seed + 1)
 
 
+@pytest.mark.parametrize("K,tau", [(4, 1), (4, 4), (8, 2)])
+def test_paper_setting_small_cnn(B, torch, K, tau):
+    # the paper's own experiment shape (Sec. VI-VII): its two-convolution digit classifier
+    # (1,199,882 parameters), 4 or 8 workers, tau in {1, 2, 4}, communication suppressed one
+    # third of the time, alpha = 0.1, dynamic weights; 60 rounds at full size
+    layout = W.mnist_cnn_layout()
+    assert W.total_params(layout) == 1_199_882
+    cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=60, tau=tau,
+                    p_fail=1 / 3, alpha=0.1)
+    _check_run(B, cfg, _layout_inputs(layout, K))
+
+
 def test_config_resnet18_shape_reduced(B, torch):
     # ResNet-18-shaped layout at 1/8 width (62 tensors, ragged tail), K=8, tau=4,
     # Bernoulli(0.1) communication failures, 200 rounds
