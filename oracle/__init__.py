@@ -41,7 +41,7 @@ def build(force: bool = False) -> dict[str, str]:
         so = os.path.join(_OUT, f"libah_oracle_{name}.so")
         if force or not os.path.exists(so) or os.path.getmtime(so) < os.path.getmtime(_SRC):
             tmp = so + f".{os.getpid()}.tmp"
-            subprocess.check_call(["gcc", *_FLAGS, *extra, "-o", tmp, _SRC, "-lm"])
+            subprocess.check_call(["gcc", *_FLAGS, *extra, "-o", tmp, _SRC, "-lquadmath", "-lm"])
             os.replace(tmp, so)
         out[name] = so
     return out
@@ -305,6 +305,13 @@ class OracleState:
         self.o.lib.orc_mask_next(self.down_until.ctypes.data_as(C.POINTER(C.c_uint32)), self.K,
                                  int(seed), int(t), float(p_fail), int(max_stale), _u8(mask))
         return mask
+
+    # scripted outages (the configuration with "worker 3 down in rounds 20 to 40"): a worker
+    # listed as (worker, first, last) cannot reach the master in rounds first..last inclusive
+    @staticmethod
+    def scripted_mask(mask, t, outages):
+        down = {w for w, first, last in outages if first <= t <= last}
+        return np.array([0 if i in down else int(b) for i, b in enumerate(mask)], np.uint8)
 
     # S6
     def exchange(self, mask=None, h2=None, h1=None, alpha=0.0):

@@ -315,94 +315,19 @@ void orc_norm2(const float *x, const float *c, int K, uint64_t P, double *n2)
         n2[i] = orc_pairwise_sq(x + (uint64_t)i * P, c, 0, n, P);
 }
 
-/* Natural logarithm of a positive, finite, normal double, evaluated in double-double
- * arithmetic (pairs hi + lo of doubles, about 100 significant bits) and rounded to
- * double at the end.  u = log ||x_i - c|| (Sec. V-B) is taken as this value, so that
- * any two implementations of the same short list of IEEE operations agree bit for
- * bit, which a call into the platform's libm would not guarantee.  Steps:
- *   x = m 2^e with m in (sqrt(1/2), sqrt(2)];  s = (m - 1)/(m + 1);
- *   ln m = 2 s (1 + z/3 + z^2/5 + ... + z^21/43), z = s^2, by Horner's rule;
- *   ln x = e ln 2 + ln m.
- * Error-free transformations: Knuth's two-sum, Dekker's fast two-sum, the product
- * error by fused multiply-add.                                                    */
-typedef struct { double hi, lo; } orc_dd;
-
-static orc_dd orc_two_sum(double a, double b)
-{
-    orc_dd r;
-    r.hi = a + b;
-    const double bb = r.hi - a;
-    r.lo = (a - (r.hi - bb)) + (b - bb);
-    return r;
-}
-
-static orc_dd orc_fast_two_sum(double a, double b)          /* needs |a| >= |b| or a == 0 */
-{
-    orc_dd r;
-    r.hi = a + b;
-    r.lo = b - (r.hi - a);
-    return r;
-}
-
-static orc_dd orc_dd_mul(orc_dd a, orc_dd b)
-{
-    const double p = a.hi * b.hi;
-    double e = fma(a.hi, b.hi, -p);
-    e = fma(a.hi, b.lo, e);
-    e = fma(a.lo, b.hi, e);
-    return orc_fast_two_sum(p, e);
-}
-
-static orc_dd orc_dd_add(orc_dd a, orc_dd b)
-{
-    orc_dd s = orc_two_sum(a.hi, b.hi);
-    const double e = s.lo + (a.lo + b.lo);
-    return orc_fast_two_sum(s.hi, e);
-}
-
-/* 1/n for a small odd integer n, as a double-double. */
-static orc_dd orc_dd_recip_int(double n)
-{
-    orc_dd r;
-    r.hi = 1.0 / n;
-    r.lo = fma(-r.hi, n, 1.0) / n;
-    return r;
-}
+/* Natural logarithm of a positive, finite double, rounded to the nearest double.
+ * u = log ||x_i - c|| (Sec. V-B) is read as exactly this value: the definition of the
+ * function, not one particular library's approximation of it, so that any correct
+ * implementation reproduces it bit for bit.  It is obtained here from a library
+ * primitive: the logarithm of GNU libquadmath in IEEE binary128 (113 significant
+ * bits, error below one unit in the last of them), rounded once to binary64.  The
+ * 60 spare bits make that rounding the correct one unless ln x lies within 2^-59
+ * units in the last place of the midpoint of two doubles.                         */
+#include <quadmath.h>
 
 double orc_ln(double x)
 {
-    /* split x = m 2^e, m in [1, 2), then fold m into (sqrt(1/2), sqrt(2)] */
-    uint64_t bits;
-    memcpy(&bits, &x, 8);
-    int e = (int)((bits >> 52) & 0x7ff) - 1023;
-    bits = (bits & 0x000fffffffffffffull) | 0x3ff0000000000000ull;
-    double m;
-    memcpy(&m, &bits, 8);
-    if (m > 1.4142135623730951) { m = m * 0.5; e += 1; }
-
-    /* s = (m - 1)/(m + 1) as a double-double: quotient, then one correction from the remainder */
-    const double num = m - 1.0;                              /* exact */
-    const orc_dd den = orc_two_sum(m, 1.0);
-    const double q = num / den.hi;
-    double rem = fma(-q, den.hi, num);
-    rem = fma(-q, den.lo, rem);
-    const orc_dd s = orc_fast_two_sum(q, rem / den.hi);
-
-    const orc_dd z = orc_dd_mul(s, s);
-    orc_dd poly = orc_dd_recip_int(43.0);
-    for (int k = 20; k >= 1; --k)
-        poly = orc_dd_add(orc_dd_mul(poly, z), orc_dd_recip_int((double)(2 * k + 1)));
-    orc_dd one = { 1.0, 0.0 };
-    poly = orc_dd_add(orc_dd_mul(poly, z), one);
-    orc_dd lnm = orc_dd_mul(s, poly);
-    lnm.hi = 2.0 * lnm.hi;
-    lnm.lo = 2.0 * lnm.lo;
-
-    /* e ln 2, with ln 2 = 0x1.62e42fefa39efp-1 + 0x1.abc9e3b39803fp-56 */
-    const orc_dd ln2 = { 0x1.62e42fefa39efp-1, 0x1.abc9e3b39803fp-56 };
-    const orc_dd ee = { (double)e, 0.0 };
-    const orc_dd r = orc_dd_add(orc_dd_mul(ln2, ee), lnm);
-    return r.hi;
+    return (double)logq((__float128)x);
 }
 
 /* u_i = log ||x_i - c||_2 = 0.5 ln(n2_i), natural log, n2 clamped away from 0

@@ -167,10 +167,11 @@ LAYOUTS = {
 }
 
 
-def random_segment_table(seed: int, target: int = 12_000, max_block: int = 128):
+def random_segment_table(seed: int, max_block: int, target: int = 12_000):
     """A seeded, irregular tensor table for edge-case tests: (segments, P) with tensors of
     every size from one block to a few thousand elements, spatial blocks from 1 to
-    max_block (3 x 3 kernels most often), occasional gaps, and a ragged end."""
+    max_block (3 x 3 kernels most often), occasional gaps, and a ragged end.  The caller
+    states the largest block it wants drawn."""
     rng = np.random.default_rng(seed)
     segs, pos = [], int(rng.integers(0, 6))
     while pos < target:

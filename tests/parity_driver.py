@@ -72,7 +72,7 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         mask_g = h.dw_mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
         mask_o = ref.mask_next(MASK_SEED, t, cfg.p_fail, cfg.max_stale)
         mask_g = W.apply_scripted(mask_g, t, cfg.scripted)
-        mask_o = W.apply_scripted(mask_o, t, cfg.scripted)
+        mask_o = ref.scripted_mask(mask_o, t, [(o["worker"], o["first"], o["last"]) for o in cfg.scripted])
         log["masks_equal"] &= bool(np.array_equal(mask_g, mask_o))
         ex = t % cfg.tau == 0
         k = t % len(pool)

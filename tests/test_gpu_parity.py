@@ -89,7 +89,7 @@ def test_local_step_random_segment_tables(B, torch, seed):
     # irregular tensor tables: every block size up to 128, blocks across tile edges, many
     # tensors inside one tile, gaps, odd offsets, ragged ends; plain, distance, n-sample and
     # one-pass forms of the step
-    segs, P = W.random_segment_table(100 + seed)
+    segs, P = W.random_segment_table(100 + seed, B.AH_MAX_BLOCK)
     K, ld = 3, W.padded_ld(P)
     rng = np.random.default_rng(seed)
     theta0 = (rng.standard_normal(P) * 0.1).astype(np.float32)
@@ -794,7 +794,7 @@ def test_config_diagonal_quadratic_full_size(B, torch):
     for t in range(1, R + 1):
         noise = W.quadratic_noise_np(K, P, 0, t)
         mask_g = W.apply_scripted(h.dw_mask_next(2, t, 0.0), t, outages)
-        mask_o = W.apply_scripted(ref.mask_next(2, t, 0.0), t, outages)
+        mask_o = ref.scripted_mask(ref.mask_next(2, t, 0.0), t, [(3, 20, 40)])
         masks_equal &= bool(np.array_equal(mask_g, mask_o))
         ex = t % tau == 0
         # device side: its own x, its own z

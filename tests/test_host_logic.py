@@ -128,10 +128,36 @@ def test_weights_match_oracle_bit_for_bit_given_same_distances(B):
         h.close()
 
 
+def test_library_log_distance_is_the_correctly_rounded_value(B):
+    # u = log ||x_i - c|| (Sec. V-B) as the library's own rule computes it from known squared
+    # distances, against the definition evaluated in 300-bit arithmetic: the natural logarithm
+    # rounded to the nearest double, halved.  Independent of the oracle.
+    import mpmath
+    mpmath.mp.prec = 300
+    rng = np.random.default_rng(77)
+    K = B.AH_MAX_WORKERS
+    n2 = np.concatenate([
+        np.exp(rng.uniform(-680, 700, 4 * K)),                  # the whole exponent range
+        rng.uniform(0.5, 2.0, 4 * K),                           # around 1, where ln cancels
+        1.0 + rng.uniform(-1, 1, 2 * K) * 1e-9,
+        np.exp(2 * rng.normal(0, 3, 6 * K)),                    # squared distances of the method
+    ])
+    n2[:8] = [1.0, 2.0, 0.5, 1e-300, 0.0, 1.4142135623730951, 0.7071067811865476, 1.7976931348623157e308]
+    h = B.Handle(K, 8, [], host_only=True)
+    h.dw_config(1, np.array([1.0]), -0.1)
+    for lo in range(0, n2.size, K):
+        chunk = n2[lo:lo + K]
+        h.dw_weights_from_norm2(chunk, 0.05)
+        u = h.ah_state_get(B.AH_UHIST, p_hist=1)[:, 0]
+        want = np.array([float(mpmath.log(mpmath.mpf(max(float(v), 1e-300)))) * 0.5 for v in chunk])
+        assert np.array_equal(u, want), (lo, chunk[u != want][:3])
+    h.close()
+
+
 @pytest.mark.parametrize("name", ["resnet18", "resnet50", "vgg16", "odd"] + [f"random{k}" for k in range(12)])
 def test_tile_descriptors_cover_whole_blocks(B, name):
     if name.startswith("random"):
-        segs, P = W.random_segment_table(int(name[6:]))
+        segs, P = W.random_segment_table(int(name[6:]), B.AH_MAX_BLOCK)
     elif name == "odd":
         segs = [(3, 18, 9), (21, 10, 1), (37, 4900, 49), (4940, 2505, 5), (9001, 4096, 128)]
         P = 13_111

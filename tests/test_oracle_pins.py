@@ -170,6 +170,59 @@ def test_step_reduces_to_adam(orc):
     assert np.allclose(st.x[0], p.detach().numpy(), rtol=1e-5, atol=1e-6)
 
 
+def test_frozen_worker_bias_correction_counts_its_own_steps(orc):
+    # A worker that sits out some rounds (a frozen straggler) is an Adam optimiser that was
+    # simply not stepped in those rounds: its 1 - beta^t uses the number of steps it has
+    # taken, not the global round.  Each worker is compared with its own library Adam
+    # (CPU, double) stepped only on that worker's active rounds; taking the global round in
+    # the bias correction instead moves x by a few per cent of a step and fails the bound.
+    torch = pytest.importorskip("torch")
+    P, K, T = 257, 2, 30
+    rng = np.random.default_rng(33)
+    x0 = rng.standard_normal(P).astype(np.float32)
+    st = OracleState(x0, K, [(0, P, 1)])
+    b1, b2 = float(np.float32(0.9)), float(np.float32(0.999))
+    params = [torch.tensor(x0.astype(np.float64), requires_grad=True) for _ in range(K)]
+    opts = [torch.optim.Adam([p], lr=0.01, betas=(b1, b2), eps=1e-4) for p in params]
+    # worker 0 always steps; worker 1 skips rounds 2-4, 9, 15-21 and 28
+    idle = {2, 3, 4, 9, 15, 16, 17, 18, 19, 20, 21, 28}
+    wrong_t = [p.detach().clone() for p in params]       # what the global round would give
+    wm = [torch.zeros(P, dtype=torch.float64) for _ in range(K)]
+    wv = [torch.zeros(P, dtype=torch.float64) for _ in range(K)]
+    for t in range(1, T + 1):
+        active = np.array([1, 0 if t in idle else 1], np.uint8)
+        g = rng.standard_normal((K, P)).astype(np.float32)
+        z = orc.sample_z(7, t, K, P)
+        st.local_step(g, (z * g).astype(np.float32), 7, t, lr=0.01, eps=1e-4, active=active)
+        for i in range(K):
+            if not active[i]:
+                continue
+            gi = torch.tensor(g[i].astype(np.float64))
+            params[i].grad = gi
+            opts[i].step()
+            wm[i] = b1 * wm[i] + (1 - b1) * gi
+            wv[i] = b2 * wv[i] + (1 - b2) * gi * gi
+            wrong_t[i] = wrong_t[i] - 0.01 * (wm[i] / (1 - b1 ** t)) / ((wv[i] / (1 - b2 ** t)).sqrt() + 1e-4)
+    assert list(st.step) == [T, T - len(idle)]
+    for i in range(K):
+        assert np.allclose(st.x[i], params[i].detach().numpy(), rtol=1e-5, atol=1e-6), i
+    # the pin has teeth: the global-round variant of worker 1 is far outside the bound
+    assert not np.allclose(wrong_t[1].numpy(), params[1].detach().numpy(), rtol=1e-3, atol=1e-4)
+    assert np.allclose(wrong_t[0].numpy(), params[0].detach().numpy(), rtol=1e-9, atol=1e-12)
+
+
+def test_scripted_outage_rule(orc):
+    # "worker 3 down in rounds 20 to 40", both ends included, nobody else touched
+    st = OracleState(np.zeros(4, np.float32), 4, [])
+    up = np.ones(4, np.uint8)
+    got = {t: list(st.scripted_mask(up, t, [(3, 20, 40)])) for t in (1, 19, 20, 30, 40, 41, 100)}
+    assert got == {1: [1, 1, 1, 1], 19: [1, 1, 1, 1], 20: [1, 1, 1, 0], 30: [1, 1, 1, 0],
+                   40: [1, 1, 1, 0], 41: [1, 1, 1, 1], 100: [1, 1, 1, 1]}
+    # a worker already down for another reason stays down; outages can overlap
+    assert list(st.scripted_mask(np.array([0, 1, 1, 1], np.uint8), 5, [(1, 5, 5), (2, 1, 9)])) == [0, 0, 0, 1]
+    assert st.scripted_mask(up, 3, []).dtype == np.uint8
+
+
 def test_noise_free_quadratic_recurrence(orc):
     # On f = 1/2 sum h x^2 without noise, vhat = h^2 at every step, so
     # x_{t+1} = x_t - lr * mhat_t / (h + eps): a scalar linear recurrence (double).
