@@ -77,8 +77,46 @@ def test_static_scratch_rejects_what_does_not_fit():
                                    stream) == B.AH_ERR_ALIGN
     assert lib.ah_distances_static(None, 1024, buf.data_ptr(), 2, 1024, out.data_ptr(),
                                    stream) == B.AH_ERR_INVALID_ARG
-    # and the largest size that fits still runs
+    # a small call still runs after the refusals (x == c: every distance is zero)
     assert lib.ah_distances_static(buf.data_ptr(), 1024, buf.data_ptr(), 4, 1024, out.data_ptr(),
                                    stream) == B.AH_OK
     torch.cuda.synchronize()
     assert np.all(out[:4].cpu().numpy() == 0.0)
+
+
+def test_static_scratch_at_exactly_its_capacity_and_one_entry_above():
+    """K = 128 workers of 2^20 parameters need 128 x 1024 tile sums: every entry of the
+    built-in array.  The result must still equal the handle path bit for bit, twice in a
+    row; one worker more, or one tile more per worker, is refused."""
+    import torch
+    from paper_2409_09242_b200 import binding as B
+    torch.cuda.set_device(0)
+    K, P = 128, 1 << 20
+    assert K * (P // 1024) == B.AH_STATIC_SCRATCH_ENTRIES
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    cd = torch.empty(P, device="cuda").normal_(generator=gen)
+    xd = cd[None, :] + torch.empty((K, P), device="cuda").normal_(generator=gen) * 0.02
+    # the handle path on the same device arrays
+    h = B.Handle(K, P, [])
+    h.ah_state_set(B.AH_CENTER, cd)
+    h.ah_state_set(B.AH_X, xd)
+    z = torch.zeros((K, P), device="cuda")                       # never read: nobody steps
+    h.ah_local_step(z, z, 1, lr=0.0, active=np.zeros(K, np.uint8), want_dist=True)
+    want = h.ah_state_get(B.AH_NORM2).copy()
+    h.close()
+    out = torch.empty(K + 1, dtype=torch.float64, device="cuda")
+    for call in range(2):
+        out.fill_(-1.0)
+        B.ah_distances_static(xd, cd, out)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        assert np.array_equal(got[:K], want), call
+        assert got[K] == -1.0                                     # nothing written past K
+    assert np.all(want > 0) and np.allclose(want, P * 0.02 ** 2, rtol=0.05)
+    lib = B.raw()
+    stream = torch.cuda.current_stream().cuda_stream
+    # one tile more per worker rounds up to 2048 tiles; one worker more needs 129 x 1024
+    assert lib.ah_distances_static(xd.data_ptr(), P + 4, cd.data_ptr(), K, P + 4, out.data_ptr(),
+                                   stream) == B.AH_ERR_TOO_LARGE
+    assert lib.ah_distances_static(xd.data_ptr(), P, cd.data_ptr(), K + 1, P, out.data_ptr(),
+                                   stream) == B.AH_ERR_TOO_LARGE
