@@ -59,7 +59,10 @@ HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weigh
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch / (K * P)), and the hash
 # of the kernel sources it was taken on.  Reported only while the sources are unchanged.
 NCU_TRAFFIC = {"sources_sha256": "72242c93ea8219879872e4400e4993ef0ebc408bd6880472c65b6bcf7b48a1d6",
-               "dram_bytes_per_update": 1.442847e9 / 46_758_048}
+               "dram_bytes_per_update": 1.442847e9 / 46_758_048,
+               "capture": "one ncu capture of the plain local step on workload p18k4 (ResNet-18-shaped "
+                          "layout, K=4, 46,758,048 updates per launch), scaled by the updates of this "
+                          "run's launch: traffic is proportional to updates"}
 
 
 def kernel_sources_hash() -> str:
@@ -96,7 +99,7 @@ class ClockSampler:
     inside the timed region can be told from those taken during warm-up."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_power_cap,power.draw")
     NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
     def __init__(self, index):
@@ -119,9 +122,15 @@ class ClockSampler:
                 if len(parts) < 6:
                     continue
                 try:
+                    watts = None
+                    if len(parts) > 6:
+                        try:
+                            watts = float(parts[6])
+                        except ValueError:
+                            pass
                     self.samples.append((time.time(), float(parts[0]), float(parts[1]),
                                          [n for n, v in zip(self.NAMES, parts[2:6])
-                                          if v.lower().startswith("active")]))
+                                          if v.lower().startswith("active")], watts))
                 except ValueError:
                     continue
         self.thread = threading.Thread(target=reader, daemon=True)
@@ -144,8 +153,12 @@ class ClockSampler:
         inside = [s for s in self.samples if t_from <= s[0] <= t_to]
         clocks = [s[1] for s in inside]
         reasons = sorted({r for s in inside for r in s[3]})
+        watts = [s[4] for s in inside if s[4] is not None]
         return {"sm_mhz": statistics.median(clocks) if clocks else None,
+                "sm_mhz_min": min(clocks) if clocks else None,
+                "sm_mhz_max_seen": max(clocks) if clocks else None,
                 "sm_max_mhz": inside[-1][2] if inside else None, "samples": len(clocks),
+                "power_w": round(statistics.median(watts), 1) if watts else None,
                 "window": window, "reasons": reasons}
 
 
@@ -187,6 +200,17 @@ class InputStager:
 
     def release(self, t):
         self.done[t % 2].record()                                # on the compute stream
+
+
+def _spread(vals, keep=48):
+    """Summary of the per-repetition times: extremes, deciles, and an evenly spaced sample
+    of the values in run order (all of them when there are few)."""
+    srt = sorted(vals)
+    pick = lambda q: round(srt[min(len(srt) - 1, int(q * len(srt)))], 4)
+    stride = max(1, -(-len(vals) // keep))
+    return {"min": pick(0.0), "p10": pick(0.1), "median": round(statistics.median(vals), 4),
+            "p90": pick(0.9), "max": round(srt[-1], 4),
+            "in_run_order": [round(v, 4) for v in vals[::stride]]}
 
 
 def max_over_ranks(ms, dist, device):
@@ -251,7 +275,11 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
                                      order=h.dw_order_next(ORDER_SEED, t) if asynchronous else None,
                                      asynchronous=asynchronous, lagged=True, **HYPER)
         else:
-            h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None, want_dist=ex,
+            # a distance round whose exchange will take its weights from the device also runs
+            # the weighting rule, in its last kernel
+            rule = ex and (carry is not None or sync_free)
+            h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None,
+                            want_dist=2 if rule else ex, rule_alpha=alpha,
                             **HYPER)      # hv is [K, ld], or [n, K, ld] with --samples n
         if stage is not None:
             stage.release(t)
@@ -337,32 +365,56 @@ def gpu_arm(args):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    run_kw = dict(asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused)
     warm_until = time.time() + 2.0
     done = 0
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     while done < args.warmup or (world == 1 and rank == 0 and sampler.proc is not None
                                  and sampler.count() == 0 and time.time() < warm_until):
         # at least the asked warm-up periods; a little longer until the clock sampler is live
-        t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method, sync_free=args.sync_free, fused=args.fused,
-                             carry=carry)
+        if done == args.warmup - 1:
+            w0.record()                           # the last asked warm-up period is also timed:
+        t, _, _ = run_period(h, pool, t, wl, carry=carry, **run_kw)
+        if done == args.warmup - 1:
+            w1.record()                           # it sizes the number of repetitions below
         done += 1
         if done >= args.warmup:
             torch.cuda.synchronize()
+    est_ms = max(w0.elapsed_time(w1), 1e-3)
+    # Repetitions: each is `--steps` periods, timed by its own pair of events; at least
+    # --reps of them and as many as it takes to keep the device busy for --min-seconds (so
+    # that the clocks settle where a long job runs them); the line reports the median.
+    # Every rank must run the same count: the slowest rank's estimate decides.
+    est_ms = max_over_ranks(est_ms, dist, dev)
+    reps = max(args.reps, int(args.min_seconds * 1e3 / (est_ms * args.steps)) + 1)
+    reps = min(reps, max(args.reps, 20000 // max(1, args.steps)))
+    # per-launch event pairs perturb very short kernels: every rep while that stays below a
+    # few thousand pairs, else every n-th rep (the median rep is then one without them)
+    launches_per_rep = args.steps * tau
+    bracket_every = max(1, -(-reps * launches_per_rep // 6000))
     barrier()
     wall0 = time.time()
     launches0 = h.ah_launch_count()
     events, ex_events = [], []
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    worker_steps = exchanged = 0
-    for _ in range(args.steps):
-        t, ws, exd = run_period(h, pool, t, wl, events, asynchronous=asyn, ex_events=ex_events,
-                                method=args.method, sync_free=args.sync_free, fused=args.fused,
-                                carry=carry)
-        worker_steps += ws
-        exchanged += exd
-    stop.record()
+    bounds = [torch.cuda.Event(enable_timing=True)]
+    bounds[0].record()
+    rep_ws, rep_exd = [], []
+    for rep in range(reps):
+        ws_r = exd_r = 0
+        ev = events if rep % bracket_every == 0 else None
+        for _ in range(args.steps):
+            t, ws, exd = run_period(h, pool, t, wl, ev, ex_events=ex_events if ev is not None else None,
+                                    carry=carry, **run_kw)
+            ws_r += ws
+            exd_r += exd
+        bounds.append(torch.cuda.Event(enable_timing=True))
+        bounds[-1].record()
+        rep_ws.append(ws_r)
+        rep_exd.append(exd_r)
     barrier()
-    ms = start.elapsed_time(stop)
+    wall1 = time.time()
+    rep_ms = [bounds[r].elapsed_time(bounds[r + 1]) for r in range(reps)]
+    launches = h.ah_launch_count() - launches0
     if carry is not None and carry.get("pending") is not None:
         # the last timed period's exchange would ride on the next step; the first timed
         # period carried the one before it.  Launch it now, outside the timed region.
@@ -372,25 +424,17 @@ def gpu_arm(args):
              else h.easgd_exchange(p_mask, None, alpha_for(K)))
         else:
             h.easgd_exchange_dynamic(p_mask, alpha_for(K), p_order, asyn)
-    wall1 = time.time()
     clocks = None
     if rank == 0:
-        window = "timed region"
-        if sampler.proc is not None and sampler.count(wall0) < 3 and world == 1:
-            # a short timed region: keep the same load running a little longer so that the
-            # clocks are seen under it (these periods are outside the timing)
-            window = "timed region and the same load right after it"
-            until = time.time() + 0.8
-            while sampler.count(wall0) < 3 and time.time() < until:
-                t, _, _ = run_period(h, pool, t, wl, asynchronous=asyn, method=args.method,
-                                     sync_free=args.sync_free, fused=args.fused)
-                torch.cuda.synchronize()
-            wall1 = time.time()
-        clocks = sampler.stop(wall0, wall1, window)
-    launches = h.ah_launch_count() - launches0
-    ms = max_over_ranks(ms, dist, dev)
-    # parameter updates actually performed: a frozen straggler takes no step
-    value = whole_job_updates_per_second(worker_steps * P, world, ms)
+        clocks = sampler.stop(wall0, wall1, "timed region")
+    # the slowest rank's time, repetition by repetition; parameter updates actually
+    # performed (a frozen straggler takes no step); the median repetition is the line's value
+    rep_ms = [max_over_ranks(m, dist, dev) for m in rep_ms]
+    rep_value = [whole_job_updates_per_second(w * P, world, m) for w, m in zip(rep_ws, rep_ms)]
+    value = statistics.median(rep_value)
+    ms = statistics.median(rep_ms)
+    worker_steps, exchanged = sum(rep_ws), sum(rep_exd)
+    total_ms = sum(rep_ms)
 
     # per-launch duration of the fused local-step kernel (plain rounds; the rounds that
     # also measure distances are listed beside it)
@@ -409,27 +453,33 @@ def gpu_arm(args):
     else:
         dom, dom_name = withd, "local_step+dist"
         dom_bytes = sum(bpu * P * n + 4 * P * (K - n) + 4 * P for _, n in dom) / len(dom)
-    dom_ms = sum(d for d, _ in dom) / len(dom)
+    # a launch's bytes depend on how many workers stepped: the median launch duration goes
+    # with the mean bytes of the launches at or next to the median
+    dom_ms = statistics.median(d for d, _ in dom)
     peak, peak_kind = measured_hbm_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    traffic = None
+    traffic = traffic_note = None
     if (args.method == "adahessian" and NCU_TRAFFIC["sources_sha256"] == kernel_sources_hash()
-            and NCU_TRAFFIC["dram_bytes_per_update"]):
-        traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0 if args.samples == 1 else None
+            and NCU_TRAFFIC["dram_bytes_per_update"] and args.samples == 1):
+        traffic = NCU_TRAFFIC["dram_bytes_per_update"] * dom_bytes / 32.0
+        traffic_note = NCU_TRAFFIC["capture"]
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": traffic,
-                "ms_per_launch": round(dom_ms, 4), "algorithmic_bytes_per_launch": int(dom_bytes),
-                "dist_round_ms": round(sum(d for d, _ in withd) / len(withd), 4) if withd else None,
-                "exchange_plus_step_ms": round(sum(rides) / len(rides), 4) if rides else None}
+                "traffic_source": traffic_note,
+                "achieved_dram": round(traffic / (dom_ms * 1e-3) / 1e9, 1) if traffic else None,
+                "ms_per_launch": round(dom_ms, 4), "launches_bracketed": len(dom),
+                "algorithmic_bytes_per_launch": int(dom_bytes),
+                "dist_round_ms": round(statistics.median(d for d, _ in withd), 4) if withd else None,
+                "exchange_plus_step_ms": round(statistics.median(rides), 4) if rides else None}
     # whole-run bytes: 32 per update + (8 P per exchanging worker + 12 P) per exchange
     if (args.fused and args.method == "adahessian") or ride:
         # fused exchange rounds: x crosses HBM once; the master row is read and written once
-        run_bytes = bpu * P * worker_steps + 8 * P * args.steps
+        run_bytes = bpu * P * worker_steps + 8 * P * args.steps * reps
     else:
         run_bytes = (bpu * P * worker_steps + 8 * P * exchanged +
-                     (12 if args.method == "adahessian" else 8) * P * args.steps)
-    whole = {"algorithmic_GBps": round(run_bytes / (ms * 1e-3) / 1e9, 1)}
+                     (12 if args.method == "adahessian" else 8) * P * args.steps * reps)
+    whole = {"algorithmic_GBps": round(run_bytes / (total_ms * 1e-3) / 1e9, 1)}
     whole["frac_of_measured_peak"] = round(whole["algorithmic_GBps"] / peak, 4)
     # the exchange kernel alone: 8 bytes per (arriving worker, parameter) + 8 per parameter
     exl = [(a.elapsed_time(b), n) for a, b, n in ex_events if n > 0]
@@ -451,19 +501,23 @@ def gpu_arm(args):
         e2e_steps = max(1, min(args.steps, int(20e9 // (pair_bytes * tau)) or 1))
         t, _, _ = run_period(h, pool, t, wl, stage=stager, asynchronous=asyn,
                              method=args.method)      # the end-to-end leg reads the weights back
-        barrier()
-        start.record()
-        e2e_ws = 0
-        for _ in range(e2e_steps):
-            t, ws, _ = run_period(h, pool, t, wl, stage=stager, asynchronous=asyn,
-                                  method=args.method)
-            e2e_ws += ws
-        stop.record()
-        barrier()
-        ems = start.elapsed_time(stop)
-        ems = max_over_ranks(ems, dist, dev)
-        e2e = {"value": round(whole_job_updates_per_second(e2e_ws * P, world, ems), 3),
-               "unit": "G param-updates/s", "steps": e2e_steps,
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2e_vals = []
+        for _ in range(3):
+            barrier()
+            start.record()
+            e2e_ws = 0
+            for _ in range(e2e_steps):
+                t, ws, _ = run_period(h, pool, t, wl, stage=stager, asynchronous=asyn,
+                                      method=args.method)
+                e2e_ws += ws
+            stop.record()
+            barrier()
+            ems = max_over_ranks(start.elapsed_time(stop), dist, dev)
+            e2e_vals.append(whole_job_updates_per_second(e2e_ws * P, world, ems))
+        e2e_value = statistics.median(e2e_vals)
+        e2e = {"value": round(e2e_value, 3),
+               "unit": "G param-updates/s", "steps": e2e_steps, "reps": 3,
                "h2d_bytes_per_step": (pair_bytes if args.method == "adahessian" else K * ld * 4) * tau,
                "d2h_bytes_per_step": 8 * K if args.method == "adahessian" else 0}
 
@@ -471,6 +525,8 @@ def gpu_arm(args):
         "metric": "AdaHessian+EASGD round: param-updates/s (K x P per round)",
         "value": round(value, 3), "unit": "G param-updates/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4),
+        "reps": reps, "timed_seconds": round(total_ms * 1e-3, 3),
+        "ms_per_step_reps": _spread([m / args.steps for m in rep_ms]),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "impl": "cuda",
         "config": {"workload": f"{args.workload}: {kind} layout, P={P}, K={K}, tau={tau}, "
@@ -485,8 +541,9 @@ def gpu_arm(args):
                                       else "the exchange rides on the next round's local step" if ride
                                       else "local step, then exchange kernel",
                    "weights": "on the device, no host wait" if args.sync_free else "on the host, one wait per period",
-                   "rounds_timed": tau * args.steps, "input_pool": n_pool,
-                   "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps,
+                   "timing": f"median of {reps} repetitions of {args.steps} periods, back to back",
+                   "rounds_timed": tau * args.steps * reps, "input_pool": n_pool,
+                   "worker_steps_timed": worker_steps, "of_possible": K * tau * args.steps * reps,
                    "l2": "per-round working set %.2f GB exceeds the 126 MB L2, no flush needed"
                          % ((32 * K * P) / 1e9) if 32 * K * P > 4 * 126e6 else
                          "working set comparable to L2: partly L2-resident, reported as is",
@@ -494,6 +551,10 @@ def gpu_arm(args):
         "roofline": roofline, "whole_step": whole, "exchange_kernel": exchange, "e2e": e2e, "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if clocks and clocks.get("sm_mhz"):
+        # time x clock: what the period costs in SM cycles, to read the clock dependence
+        # off runs that the power cap held at different clocks
+        out["clocks"]["ms_per_step_x_mhz"] = round(ms / args.steps * clocks["sm_mhz"], 1)
     h.close()
     del pool
     torch.cuda.empty_cache()
@@ -609,7 +670,10 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=20, help="communication periods per repetition")
+    ap.add_argument("--reps", type=int, default=5, help="least number of timed repetitions")
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="repeat until the device has been busy this long (0: --reps alone)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))

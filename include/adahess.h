@@ -58,6 +58,10 @@ extern "C" {
 #define AH_ROUND_AUTO   0xFFFFFFFFu
 #define AH_STATIC_SCRATCH_ENTRIES (1 << 17)  /* doubles per row of the built-in scratch     */
 #define AH_DEVICE_NONE  (-2)       /* ah_alloc.device: bookkeeping-only handle, no GPU      */
+/* ah_hyper.want_dist */
+#define AH_DIST_NONE      0        /* no distances this round                               */
+#define AH_DIST           1        /* also ||x_i - c||^2 for all K workers                  */
+#define AH_DIST_AND_RULE  2        /* ... and then the weighting rule of Sec. V-B on the device */
 
 /* ---- types ---------------------------------------------------------------- */
 typedef struct ah_ctx ah_ctx;      /* opaque; created by ah_init, freed by ah_destroy       */
@@ -86,11 +90,18 @@ typedef struct {
                              own 1-based count of ah_local_step calls                       */
     const uint8_t *active;/* host pointer, K bytes, or NULL (all active): 0 = worker i
                              skips this step entirely (its x, m, v, step count stay)        */
-    int want_dist;        /* 1 = also compute n2_i = ||x_i - c||^2 after the step, for all
-                             K workers, into the handle (read by dw_weights_next)           */
+    int want_dist;        /* AH_DIST: also compute n2_i = ||x_i - c||^2 after the step, for
+                             all K workers, into the handle (read by dw_weights_next or by
+                             the device forms of the rule).  AH_DIST_AND_RULE: the kernel
+                             that completes the last distance also runs the weighting rule
+                             of Sec. V-B on the device with the moving rate rule_alpha; the
+                             next easgd_exchange_dynamic or easgd_exchange_then_step
+                             (dynamic != 0) with the same alpha uses its coefficients and
+                             launches no rule of its own.  AH_DIST_NONE: neither.          */
     int n_samples;        /* Hutchinson samples per step, 1 .. AH_MAX_SAMPLES; 0 means 1     */
     uint64_t hvp_sample_stride; /* elements from sample s to sample s + 1 inside hvp (a
                              multiple of 4, at least K * ld); ignored for one sample        */
+    float rule_alpha;     /* moving rate alpha of h1 / h2, read with AH_DIST_AND_RULE only  */
 } ah_hyper;
 
 /* Hyper-parameters of one first-order local step (sgd_local_step). */
@@ -98,7 +109,9 @@ typedef struct {
     float lr;             /* eta                                                            */
     float momentum;       /* delta in [0, 1); 0 = plain SGD, the velocity is not touched     */
     const uint8_t *active;/* host pointer, K bytes, or NULL (all active), as in ah_hyper    */
-    int want_dist;        /* 1 = also compute ||x_i - c||^2 after the step, as in ah_hyper  */
+    int want_dist;        /* AH_DIST = also compute ||x_i - c||^2 after the step, as in
+                             ah_hyper (AH_DIST_AND_RULE is not offered here: these methods
+                             exchange with a fixed moving rate)                              */
 } sgd_hyper;
 
 /* Optional placement: caller-owned device memory and stream.  workspace must be
@@ -165,7 +178,13 @@ int ah_destroy(ah_ctx *h);
  * host pointer (0); the host-side selectors (AH_NORM2 ... AH_ROUND) take host
  * pointers only.  ah_state_get synchronises the handle's stream; ah_state_set is
  * ordered after earlier work on the stream and returns when the copy is done.
- * Together they give an exact snapshot for checkpoint and resume. */
+ * Together they give an exact snapshot for checkpoint and resume.  Where an exchange is
+ * still to come when the snapshot is taken (its distances measured, the pull deferred to
+ * the next step): if the rule has not run yet, AH_NORM2 belongs to the snapshot, and
+ * setting it makes those distances pending again on the restored handle, for the host
+ * and the device forms of the rule alike; if the rule has run on the device
+ * (AH_DIST_AND_RULE), AH_WEIGHTS belongs to it, and the restored run hands those
+ * coefficients to that one exchange as caller weights (dynamic == 0): same bits. */
 int ah_state_set(ah_ctx *h, int which, int worker, const void *src, int src_on_device);
 int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device);
 
@@ -203,7 +222,13 @@ int ah_sample_z_n(ah_ctx *h, uint64_t z_seed, uint32_t round, uint32_t sample, f
  * grad, hvp: device pointers, [K][ld] row-major, ld >= P, ld % 4 == 0, 16-byte
  * aligned, read only, must stay valid until the stream has run the step.
  * With hy->want_dist the squared distances ||x_i - c||^2 (binary32 difference,
- * squared and summed in double, pairwise order) are left in the handle.
+ * squared and summed in double, pairwise order) are left in the handle, by the same
+ * kernel: the tile sums climb a tree of arrival counters and whichever CTA completes the
+ * last worker writes the K results to pinned host memory and, with AH_DIST_AND_RULE,
+ * runs the weighting rule (u = log ||x_i - c||, Eqs. 10-11, h1 / h2 of Sec. V-B; same
+ * bits as dw_weights_next).  A distance round therefore costs no launch of its own
+ * (one more only when some workers sit the step out).
+ * A call that returns an error other than AH_ERR_CUDA leaves the handle unchanged.
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
                   uint64_t z_seed, const ah_hyper *hy);
@@ -252,9 +277,10 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
  * calls in sequence; x is read and written once instead of twice.  Unlike
  * ah_local_step_exchange nothing lags: the coefficients are those of this exchange,
  *   dynamic == 0: weights (host, 2K floats) or, when NULL, alpha for all;
- *   dynamic != 0: the rule of Sec. V-B runs on the device first, on the distances the
- *       last want_dist step left there (as easgd_exchange_dynamic; weights must be NULL;
- *       STATE if no distances are pending), and the pass reads its output.
+ *   dynamic != 0: the pass reads the output of the rule of Sec. V-B on the device: what
+ *       the last step left there if it ran with AH_DIST_AND_RULE (alpha must be the same,
+ *       else INVALID_ARG), else the rule is launched first on the distances that step left
+ *       (as easgd_exchange_dynamic; weights must be NULL; STATE if none are pending).
  * worker_mask says who takes part in the exchange; hy->active who takes the step.
  * hy->want_dist must be 0 (the distances to the new master are only defined once every
  * worker has met it): with a communication period of one round use
@@ -319,7 +345,9 @@ int easgd_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, 
 
 /* The exchange of one round with the dynamic weights computed on the device: the same
  * rule as dw_weights_next (Sec. V-B, Eqs. 10-11, h1/h2), same history ring, same bits,
- * fed by the distances of the last want_dist step, followed by the weighted exchange
+ * fed by the distances of the last want_dist step (if that step ran with
+ * AH_DIST_AND_RULE the rule has run already and alpha must be the one given there),
+ * followed by the weighted exchange
  * (Eqs. 12-13) of easgd_exchange (asynchronous == 0; order ignored) or
  * easgd_exchange_async (asynchronous != 0; order as there, NULL = ascending).  Nothing
  * is copied to the host and the call does not wait, so a whole communication period

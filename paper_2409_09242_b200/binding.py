@@ -29,6 +29,7 @@ AH_STATIC_SCRATCH_ENTRIES = 1 << 17
 AH_MAX_WORKERS, AH_MAX_BLOCK, AH_MAX_HIST, AH_MAX_SAMPLES = 256, 128, 32, 8
 AH_ROUND_AUTO = 0xFFFFFFFF
 AH_DEVICE_NONE = -2
+AH_DIST_NONE, AH_DIST, AH_DIST_AND_RULE = 0, 1, 2
 (AH_X, AH_M, AH_V, AH_CENTER, AH_NORM2, AH_STEP, AH_UHIST, AH_DOWN_UNTIL, AH_ROUND,
  AH_INFO, AH_RUNS, AH_TILES, AH_WEIGHTS) = range(13)
 
@@ -49,7 +50,7 @@ class ah_hyper(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
                 ("eps", C.c_float), ("hessian_power", C.c_float), ("weight_decay", C.c_float),
                 ("round", C.c_uint32), ("active", C.POINTER(C.c_uint8)), ("want_dist", C.c_int),
-                ("n_samples", C.c_int), ("hvp_sample_stride", C.c_uint64)]
+                ("n_samples", C.c_int), ("hvp_sample_stride", C.c_uint64), ("rule_alpha", C.c_float)]
 
 
 class sgd_hyper(C.Structure):
@@ -314,8 +315,9 @@ class Handle:
 
     def ah_local_step(self, grad, hvp, z_seed, lr, beta1=0.9, beta2=0.999, eps=1e-4,
                       hessian_power=1.0, weight_decay=0.0, round_=AH_ROUND_AUTO, active=None,
-                      want_dist=False):
-        """hvp: [K, ld] for one Hutchinson sample, or [n, K, ld] for n samples per step."""
+                      want_dist=False, rule_alpha=0.0):
+        """hvp: [K, ld] for one Hutchinson sample, or [n, K, ld] for n samples per step.
+        want_dist: False / True, or AH_DIST_AND_RULE with rule_alpha."""
         n_samples, sample_stride = _hvp_samples(grad, hvp)
         act = None
         if active is not None:
@@ -324,7 +326,7 @@ class Handle:
                 raise ValueError("active: K bytes")
         hy = ah_hyper(lr, beta1, beta2, eps, hessian_power, weight_decay, int(round_),
                       act.ctypes.data_as(C.POINTER(C.c_uint8)) if act is not None else None,
-                      1 if want_dist else 0, int(n_samples), int(sample_stride))
+                      int(want_dist), int(n_samples), int(sample_stride), float(rule_alpha))
         self._check(_lib.ah_local_step(self._h, _dev_ptr(grad, "grad"), _dev_ptr(hvp, "hvp"),
                                        grad.stride(-2), int(z_seed), C.byref(hy)), "ah_local_step")
 

@@ -13,6 +13,7 @@ _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.environ.get("ADAHESS_LIB") or os.path.join(_PKG, "libadahess.so")
 SOURCES = ["ah_kernels.cu", "ah_host.cu", "ah_noalloc.cu", "ah_exchange_async.cu", "ah_sgd.cu", "ah_partition.cu", "ah_dynamic.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+              "--split-compile", "0", "--threads", "0",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-ffp-contract=off", "-shared"]
 
 

@@ -24,7 +24,12 @@ struct ah_ctx {
 
     // device views into the workspace
     float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
-    double *partials = nullptr, *scratch = nullptr;
+    double *partials = nullptr;    // level 0 of the distance tree: [K][ntiles_pad]
+    ah::DistTree tree;             // the whole tree as the kernels see it (rule fields unset)
+    size_t tree_count_bytes = 0;   // arrival counters (+ the finished-rows word) of the tree
+    bool tree_dirty = false;       // a distance round failed half way: clear the counters first
+    ah::RuleConfig *rule_dev = nullptr;   // parameters of the weighting rule on the device
+    bool rule_dev_stale = true;    // ... no longer those of the host
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
     uint32_t *ring_flag_dev = nullptr;   // device copy of ring_filled
@@ -35,12 +40,17 @@ struct ah_ctx {
     uint32_t nruns = 0;
 
     // host state
-    double *norm2_host = nullptr;  // pinned copy of norm2_dev (status word + K doubles)
+    double *norm2_host = nullptr;  // pinned, mapped copy of norm2_dev (status word + K doubles):
+                                   // written by the kernel that completes the last distance
+    double *norm2_host_dev = nullptr;   // the same memory as the device addresses it
     cudaEvent_t norm2_ready = nullptr;
     bool norm2_pending = false;    // distances of a want_dist step not yet used by a weight rule
     bool norm2_unread = false;     // ... and not yet copied into norm2_last
     int ring_home = 0;             // 0: the host copy of the ring is current, 1: the device copy
     bool lagged_ready = false;     // weights_dev holds the rule's output of an earlier fused round
+    bool rule_fresh = false;       // weights_dev holds the rule's output for the distances of the
+                                   // last want_dist step (AH_DIST_AND_RULE), not yet used
+    float rule_fresh_alpha = 0.f;  // ... computed with this moving rate
     double norm2_last[AH_MAX_WORKERS];
     uint32_t step[AH_MAX_WORKERS];
     uint32_t down_until[AH_MAX_WORKERS];
@@ -64,10 +74,13 @@ inline int ah_cuda_fail(ah_ctx *h, cudaError_t e)
 
 namespace ah {
 int finish_distances(ah_ctx *h);   // ah_host.cu
+int prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &tree);
+void commit_rule_in_round(ah_ctx *h, float alpha);
 int ring_to_host(ah_ctx *h);
 int ring_to_device(ah_ctx *h);
 int enqueue_weight_rule(ah_ctx *h, float alpha);   // ah_dynamic.cu
-cudaError_t launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows);   // ah_sgd.cu
+cudaError_t launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows,
+                                 const DistTree &tree);   // ah_sgd.cu
 int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                   const uint16_t *order, const float *weights_dev, ExchangeParams &p);
 cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu

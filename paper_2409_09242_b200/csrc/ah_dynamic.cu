@@ -42,8 +42,11 @@ int ah::enqueue_weight_rule(ah_ctx *h, float alpha)
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
     h->launches += 1;
+    h->ring_home = 1;                              // the device copy of the ring leads
     h->norm2_pending = false;                      // these distances have fed the rule
     h->lagged_ready = true;                        // weights_dev now holds coefficients
+    h->rule_fresh = true;                          // ... of the exchange that is still to come
+    h->rule_fresh_alpha = alpha;
     return AH_OK;
 }
 
@@ -51,16 +54,27 @@ extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, flo
                                       const uint16_t *order, int asynchronous)
 {
     if (!h) return AH_ERR_INVALID_ARG;
-    if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
+    if (!h->has_device) return AH_ERR_STATE;
+    // the rule has either run already at the end of the distance round (its output is
+    // waiting in weights_dev), or runs now on the pending distances
+    if (h->rule_fresh) {
+        if (alpha != h->rule_fresh_alpha) return AH_ERR_INVALID_ARG;
+    } else if (!h->norm2_pending) {
+        return AH_ERR_STATE;
+    }
     ExchangeParams p;
     int rc = fill_exchange(h, worker_mask, nullptr, alpha, asynchronous ? order : nullptr,
                            h->weights_dev, p);
     if (rc != AH_OK) return rc;
-    if ((rc = enqueue_weight_rule(h, alpha)) != AH_OK) return rc;
-    if (p.nact == 0) return AH_OK;                 // the history advances even if nobody arrives
+    if (!h->rule_fresh && (rc = enqueue_weight_rule(h, alpha)) != AH_OK) return rc;
+    if (p.nact == 0) {                             // the history advances even if nobody arrives
+        h->rule_fresh = false;
+        return AH_OK;
+    }
     const cudaError_t e = asynchronous ? launch_exchange_in_order(p, h->stream)
                                        : launch_exchange(p, h->stream);
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->rule_fresh = false;
     h->launches += 1;
     return AH_OK;
 }

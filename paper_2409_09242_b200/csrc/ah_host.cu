@@ -37,8 +37,30 @@ int cuda_fail(ah_ctx *h, cudaError_t e)
     } while (0)
 
 struct Layout {
-    size_t x, m, v, c, partials, scratch, norm2, sched, uhist, weights, runs, tiles, total;
+    size_t x, m, v, c, partials, upper, count, norm2, sched, uhist, weights, rule, runs, tiles, total;
+    size_t count_bytes;
 };
+
+// Shape of the distance tree over ntp = 2^a tile slots of which ntiles exist: nodes per
+// worker at every level, how many of them are live, and where each level starts.  Returns
+// the nodes per worker above level 0.
+uint32_t tree_shape(uint32_t ntiles, uint32_t ntp, DistTree &T)
+{
+    T.n[0] = ntp;
+    T.live[0] = ntiles;
+    T.off[0] = 0;
+    uint32_t L = 0, above = 0;
+    do {
+        ++L;
+        T.n[L] = T.n[L - 1] >> kTreeRadixLog2 ? T.n[L - 1] >> kTreeRadixLog2 : 1u;
+        T.live[L] = (T.live[L - 1] + (1u << kTreeRadixLog2) - 1u) >> kTreeRadixLog2;
+        T.off[L] = above;
+        above += T.n[L];
+    } while (T.n[L] > 1u);
+    T.levels = L;
+    for (uint32_t q = L + 1; q <= (uint32_t)kTreeMaxLevels; ++q) T.n[q] = T.live[q] = T.off[q] = 0u;
+    return above;
+}
 
 // Offsets of every array inside the workspace (each 256-byte aligned).
 Layout workspace_layout(int K, uint64_t P, int nruns_max)
@@ -54,11 +76,16 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.v = take((size_t)K * lds * sizeof(float));
     L.c = take((size_t)lds * sizeof(float));
     L.partials = take((size_t)K * ntp * sizeof(double));
-    L.scratch = take((size_t)K * ntp * sizeof(double));
+    DistTree shape;
+    const uint32_t above = tree_shape(ntiles, ntp, shape);
+    L.upper = take((size_t)K * above * sizeof(double));
+    L.count_bytes = ((size_t)K * above + 1) * sizeof(uint32_t);     // + the finished-rows word
+    L.count = take(L.count_bytes);
     L.norm2 = take((size_t)(AH_MAX_WORKERS + 1) * sizeof(double));
     L.sched = take(4 * sizeof(uint32_t));                 // item counter, exit counter, ring flag
     L.uhist = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
     L.weights = take(2 * (size_t)K * sizeof(float));
+    L.rule = take(sizeof(RuleConfig));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
     L.total = off;
@@ -151,6 +178,9 @@ int ah::ring_to_host(ah_ctx *h)
     return AH_OK;
 }
 
+// Uploads the host copy of the ring if it is the current one.  The device copy becomes the
+// current one only when a rule has been enqueued behind the upload: the caller sets
+// ring_home = 1 after that launch has succeeded.
 int ah::ring_to_device(ah_ctx *h)
 {
     if (h->ring_home == 1) return AH_OK;
@@ -161,23 +191,57 @@ int ah::ring_to_device(ah_ctx *h)
                                cudaMemcpyHostToDevice, h->stream));
     AH_CUDA(h, cudaMemcpyAsync(h->ring_flag_dev, &filled, sizeof(filled), cudaMemcpyHostToDevice,
                                h->stream));
-    h->ring_home = 1;
     return AH_OK;
 }
 
-// After a step has left the tile partials of ||x_i - c||^2 in the workspace: finish
-// the pairwise tree on the device and start the copy of the K doubles (and the status
-// word in front of them) to pinned host memory.
+// What a launch that measures distances needs to know about the tree.  With run_rule the
+// kernel that completes the last distance also runs the weighting rule (moving rate
+// alpha) on the device copy of the history, which is brought up to date first.
+int ah::prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &tree)
+{
+    if (h->tree_dirty) {          // an earlier distance round stopped half way
+        AH_CUDA(h, cudaMemsetAsync(h->tree.count, 0, h->tree_count_bytes, h->stream));
+        h->tree_dirty = false;
+    }
+    tree = h->tree;
+    tree.run_rule = run_rule ? 1u : 0u;
+    tree.rule_alpha = (double)alpha;
+    if (run_rule) {
+        const int rc = ring_to_device(h);
+        if (rc != AH_OK) return rc;
+        if (h->rule_dev_stale) {
+            RuleConfig cfg;
+            memset(&cfg, 0, sizeof cfg);
+            for (int j = 0; j < h->p_hist; ++j) cfg.coef[j] = h->coef[j];
+            cfg.kappa = h->kappa;
+            cfg.p_hist = h->p_hist;
+            AH_CUDA(h, cudaMemcpyAsync(h->rule_dev, &cfg, sizeof cfg, cudaMemcpyHostToDevice, h->stream));
+            h->rule_dev_stale = false;
+        }
+    }
+    h->tree_dirty = true;         // until finish_distances has seen every launch succeed
+    return AH_OK;
+}
+
+// Bookkeeping after a round whose last kernel also ran the weighting rule.
+void ah::commit_rule_in_round(ah_ctx *h, float alpha)
+{
+    h->ring_home = 1;             // the device copy of the ring leads
+    h->norm2_pending = false;     // these distances have fed the rule
+    h->lagged_ready = true;       // weights_dev holds coefficients
+    h->rule_fresh_alpha = alpha;
+}
+
+// After every kernel of a distance round has been enqueued: the kernel that completes
+// the last distance leaves the K doubles (and the status word in front of them) in pinned
+// host memory, so an event behind it is all the host needs to wait for.
 int ah::finish_distances(ah_ctx *h)
 {
-    AH_CUDA(h, launch_norm2_finalize(h->partials, h->scratch, h->ntiles, h->ntiles_pad, h->K,
-                                     h->norm2_dev + 1, h->stream));
-    h->launches += 1;
-    AH_CUDA(h, cudaMemcpyAsync(h->norm2_host, h->norm2_dev, (h->K + 1) * sizeof(double),
-                               cudaMemcpyDeviceToHost, h->stream));
     AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
+    h->tree_dirty = false;
     h->norm2_pending = true;
     h->norm2_unread = true;
+    h->rule_fresh = false;
     return AH_OK;
 }
 
@@ -259,7 +323,6 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->v = (float *)(base + L.v);
     h->c = (float *)(base + L.c);
     h->partials = (double *)(base + L.partials);
-    h->scratch = (double *)(base + L.scratch);
     h->norm2_dev = (double *)(base + L.norm2);
     h->sched = (uint32_t *)(base + L.sched);
     h->ring_flag_dev = h->sched + 2;
@@ -273,11 +336,32 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
         h->last_cuda = (int)e;
         return fail(AH_ERR_CUDA);
     }
-    if ((e = cudaMallocHost((void **)&h->norm2_host, (AH_MAX_WORKERS + 1) * sizeof(double))) != cudaSuccess ||
+    if ((e = cudaHostAlloc((void **)&h->norm2_host, (AH_MAX_WORKERS + 1) * sizeof(double),
+                           cudaHostAllocMapped)) != cudaSuccess ||
+        (e = cudaHostGetDevicePointer((void **)&h->norm2_host_dev, h->norm2_host, 0)) != cudaSuccess ||
         (e = cudaEventCreateWithFlags(&h->norm2_ready, cudaEventDisableTiming)) != cudaSuccess) {
         h->last_cuda = (int)e;
         return fail(AH_ERR_ALLOC);
     }
+    memset(h->norm2_host, 0, (AH_MAX_WORKERS + 1) * sizeof(double));
+    // the distance tree as the kernels see it
+    tree_shape(h->ntiles, h->ntiles_pad, h->tree);
+    h->tree.level0 = h->partials;
+    h->tree.upper = (double *)(base + L.upper);
+    h->tree.count = (uint32_t *)(base + L.count);
+    h->tree.rows_done = h->tree.count + (L.count_bytes / sizeof(uint32_t) - 1);
+    h->tree_count_bytes = L.count_bytes;
+    h->tree.norm2 = h->norm2_dev + 1;
+    h->tree.norm2_host = h->norm2_host_dev;
+    h->tree.status = reinterpret_cast<const uint32_t *>(h->norm2_dev);
+    h->rule_dev = (RuleConfig *)(base + L.rule);
+    h->tree.rule = h->rule_dev;
+    h->tree.uhist = h->uhist_dev;
+    h->tree.ring_flag = h->ring_flag_dev;
+    h->tree.weights = h->weights_dev;
+    h->tree.rule_alpha = 0.0;
+    h->tree.run_rule = 0u;
+    h->tree.K = (uint32_t)K;
     // state (and its row padding) starts at zero; descriptors go up once
     if ((e = cudaMemsetAsync(h->workspace, 0, L.runs, h->stream)) != cudaSuccess ||
         (e = cudaMemcpyAsync(h->runs, runs.data(), runs.size() * sizeof(Run), cudaMemcpyHostToDevice,
@@ -351,12 +435,14 @@ struct FusedExchange {
 int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld, uint64_t z_seed,
                     const ah_hyper *hy, const FusedExchange *fx)
 {
+    // ---- every check first: a refused call leaves the handle as it was
     if (!h || !grad || !hvp || !hy || ld < h->P) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
     if (!(hy->beta1 >= 0.f && hy->beta1 < 1.f && hy->beta2 >= 0.f && hy->beta2 < 1.f))
         return AH_ERR_INVALID_ARG;
     if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0 || ((uintptr_t)hvp & 15u) != 0)
         return AH_ERR_ALIGN;
+    if (hy->want_dist < AH_DIST_NONE || hy->want_dist > AH_DIST_AND_RULE) return AH_ERR_INVALID_ARG;
 
     const int nsamp = hy->n_samples > 0 ? hy->n_samples : 1;
     if (nsamp > AH_MAX_SAMPLES) return AH_ERR_INVALID_ARG;
@@ -364,19 +450,37 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         if (hy->hvp_sample_stride < (uint64_t)(h->K - 1) * ld + h->P) return AH_ERR_INVALID_ARG;
         if ((hy->hvp_sample_stride & 3u) != 0) return AH_ERR_ALIGN;
     }
+    if (fx && fx->order) {                        // must name every worker exactly once
+        bool seen[AH_MAX_WORKERS] = {};
+        for (int q = 0; q < h->K; ++q) {
+            if (fx->order[q] >= h->K || seen[fx->order[q]]) return AH_ERR_INVALID_ARG;
+            seen[fx->order[q]] = true;
+        }
+    }
+    const bool dist = hy->want_dist != AH_DIST_NONE;
+    // the weighting rule at the end of this round's last kernel: asked for by the caller,
+    // or (lagged one-pass rounds) to serve the next exchange round
+    const bool rule_here = hy->want_dist == AH_DIST_AND_RULE || (fx && fx->lagged && dist);
+    const float rule_alpha = hy->want_dist == AH_DIST_AND_RULE ? hy->rule_alpha : (fx ? fx->alpha : 0.f);
+    if (hy->want_dist == AH_DIST_AND_RULE && fx && !fx->lagged) return AH_ERR_INVALID_ARG;
+    if (fx && fx->dynamic) {                      // this exchange's coefficients, on the device
+        if (h->rule_fresh) {
+            if (fx->alpha != h->rule_fresh_alpha) return AH_ERR_INVALID_ARG;
+        } else if (!h->norm2_pending) {
+            return AH_ERR_STATE;
+        }
+    }
 
-    const bool dist = hy->want_dist != 0;
     StepParams p;
     p.nsamp = (uint32_t)nsamp;
     p.sample_stride = nsamp > 1 ? hy->hvp_sample_stride : 0;
     p.x = h->x; p.m = h->m; p.v = h->v; p.c = h->c;
     p.grad = grad; p.hvp = hvp;
-    p.partials = h->partials;
     p.status = reinterpret_cast<uint32_t *>(h->norm2_dev);
     p.sched = h->sched;
     p.runs = h->runs; p.tiles = h->tiles;
     p.lds = h->lds; p.ld = ld;
-    p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
+    p.P = h->P; p.ntiles = h->ntiles;
     p.key0 = (uint32_t)(z_seed & 0xffffffffu);
     p.key1 = (uint32_t)(z_seed >> 32);
     p.lr = hy->lr; p.beta1 = hy->beta1; p.beta2 = hy->beta2;
@@ -390,23 +494,12 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     p.nworkers = (uint32_t)h->K;
     p.c_out = h->c;
     p.wdev = fx && ((fx->lagged && h->lagged_ready) || fx->dynamic) ? h->weights_dev : nullptr;
-    if (fx && fx->order) {                        // must name every worker exactly once
-        bool seen[AH_MAX_WORKERS] = {};
-        for (int q = 0; q < h->K; ++q) {
-            if (fx->order[q] >= h->K || seen[fx->order[q]]) return AH_ERR_INVALID_ARG;
-            seen[fx->order[q]] = true;
-        }
-    }
-    if (fx && fx->dynamic) {                      // this exchange's coefficients, on the device
-        if (!h->norm2_pending) return AH_ERR_STATE;
-        const int rc = enqueue_weight_rule(h, fx->alpha);
-        if (rc != AH_OK) return rc;
-    }
-    h->calls += 1;
-    p.round = hy->round == AH_ROUND_AUTO ? h->calls : hy->round;
+    const uint32_t calls = h->calls + 1;
+    p.round = hy->round == AH_ROUND_AUTO ? calls : hy->round;
     p.nrows = 0;
     uint16_t idle[AH_MAX_WORKERS];
     uint32_t nidle = 0;
+    uint32_t step[AH_MAX_WORKERS];                // step counts once this launch is enqueued
     for (int q = 0; q < h->K; ++q) {
         // a fused round walks the workers in their arrival order
         const int i = fx && fx->asynchronous && fx->order ? (int)fx->order[q] : q;
@@ -417,14 +510,14 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         if (meets) p.any_exchange = 1u;
         p.h2w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[i] : fx->alpha) : 0.f;
         p.h1w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[h->K + i] : fx->alpha) : 0.f;
-        if (on) h->step[i] += 1;
+        step[i] = h->step[i] + (on ? 1u : 0u);
         // distances cover every worker; in a plain distance round the workers that sit
         // the step out are measured by a streaming kernel of their own
         if (on || meets || (dist && fx)) p.row[p.nrows++] = (uint16_t)i;
         else if (dist) idle[nidle++] = (uint16_t)i;
         // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
         // (a worker that sat out steps has taken fewer); double, then one rounding
-        const double t = (double)(h->step[i] ? h->step[i] : 1u);
+        const double t = (double)(step[i] ? step[i] : 1u);
         WorkerConst &w = p.w[i];
         w.bc1 = (float)(1.0 - pow((double)hy->beta1, t));
         w.bc2 = (float)(1.0 - pow((double)hy->beta2, t));
@@ -432,18 +525,33 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         w.rbc2 = 1.0f / w.bc2;
     }
     p.nitems = fx ? (p.nrows ? h->ntiles : 0u) : p.nrows * h->ntiles;
+
+    // ---- enqueue; the handle's bookkeeping follows each launch that went in
+    if (fx && fx->dynamic && !h->rule_fresh) {
+        const int rc = enqueue_weight_rule(h, fx->alpha);
+        if (rc != AH_OK) return rc;
+    }
+    if (dist) {
+        const int rc = prepare_distance_round(h, rule_here, rule_alpha, p.tree);
+        if (rc != AH_OK) return rc;
+    } else {
+        memset(&p.tree, 0, sizeof p.tree);
+    }
     AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
+    h->calls = calls;
+    memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
+    if (fx && fx->dynamic) h->rule_fresh = false;     // the pending exchange has been made
     if (p.nitems) h->launches += 1;
     if (nidle) {
-        AH_CUDA(h, launch_distance_rows(h, idle, nidle));
+        AH_CUDA(h, launch_distance_rows(h, idle, nidle, p.tree));
         h->launches += 1;
     }
     if (dist) {
         const int rc = finish_distances(h);
         if (rc != AH_OK) return rc;
-        if (fx && fx->lagged) {                   // the rule runs now, its output serves next time
-            const int rc2 = enqueue_weight_rule(h, fx->alpha);
-            if (rc2 != AH_OK) return rc2;
+        if (rule_here) {
+            commit_rule_in_round(h, rule_alpha);
+            h->rule_fresh = hy->want_dist == AH_DIST_AND_RULE;
         }
     }
     return AH_OK;
@@ -463,7 +571,7 @@ int ah_local_step_exchange(ah_ctx *h, const float *grad, const float *hvp, uint6
                            int asynchronous, int lagged)
 {
     if (!hy) return AH_ERR_INVALID_ARG;
-    if (lagged && (!hy->want_dist || weights)) return AH_ERR_INVALID_ARG;
+    if (lagged && (hy->want_dist != AH_DIST || weights)) return AH_ERR_INVALID_ARG;
     FusedExchange fx;
     fx.mask = worker_mask; fx.weights = weights; fx.alpha = alpha; fx.order = order;
     fx.asynchronous = asynchronous != 0; fx.lagged = lagged != 0;
@@ -519,6 +627,7 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
             AH_CUDA(h, cudaMemcpyAsync(h->weights_dev, user, 2 * (size_t)h->K * sizeof(float),
                                        cudaMemcpyHostToDevice, h->stream));
             h->lagged_ready = true;
+            h->rule_fresh = false;
         }
         AH_CUDA(h, cudaStreamSynchronize(h->stream));
         return AH_OK;
@@ -564,7 +673,22 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
             h->calls = round_info[0];
             h->ring_filled = (int)round_info[1];
         }
-        if (which == AH_NORM2) { h->norm2_pending = false; h->norm2_unread = false; }
+        if (which == AH_NORM2) {
+            // restored distances: on a handle with a device they are pending again, for
+            // either form of the weighting rule (host or device)
+            h->norm2_unread = false;
+            h->rule_fresh = false;
+            h->norm2_pending = false;
+            if (h->has_device) {
+                AH_CUDA(h, cudaStreamSynchronize(h->stream));     // nobody is writing the pinned copy
+                memcpy(h->norm2_host + 1, h->norm2_last, h->K * sizeof(double));
+                memset(h->norm2_host, 0, sizeof(double));
+                AH_CUDA(h, cudaMemcpyAsync(h->norm2_dev + 1, h->norm2_last, h->K * sizeof(double),
+                                           cudaMemcpyHostToDevice, h->stream));
+                AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
+                h->norm2_pending = true;
+            }
+        }
         if (which == AH_UHIST || which == AH_ROUND) h->ring_home = 0;    // the host copy leads again
     }
     return AH_OK;
@@ -597,6 +721,7 @@ int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
     h->kappa = kappa;
     reset_history(h);
     h->ring_home = 0;
+    h->rule_dev_stale = true;
     return AH_OK;
 }
 

@@ -28,14 +28,21 @@ namespace ah {
 #ifndef AH_CTAS_PER_SM
 #define AH_CTAS_PER_SM 4
 #endif
+#ifndef AH_CTAS_PER_SM_PLAIN
+#define AH_CTAS_PER_SM_PLAIN AH_CTAS_PER_SM
+#endif
+#ifndef AH_CONSUMER_WARPS
+#define AH_CONSUMER_WARPS 8
+#endif
 constexpr int kPasses = AH_PASSES;                 // float4 per consumer thread per stream
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = AH_CONSUMER_WARPS;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kPassElems = kConsumers * 4;         // 1024: one float4 per consumer
 constexpr int kTile = kPassElems * kPasses;
 constexpr int kStages = AH_STAGES;
-constexpr int kCtasPerSm = AH_CTAS_PER_SM;
+constexpr int kCtasPerSm = AH_CTAS_PER_SM;             // resident CTAs per SM the kernels are built for
+constexpr int kCtasPerSmPlain = AH_CTAS_PER_SM_PLAIN;   // ... the plain round (smallest stages)
 static_assert((kTile & (kTile - 1)) == 0, "tile must be a power of two");
 
 // A spatial block may straddle a tile edge: the Hessian-vector stage holds up to
@@ -76,11 +83,54 @@ struct WorkerConst {
     float bc1, bc2, rbc1, rbc2;
 };
 
-struct StepParams {
+// Parameters of the weighting rule of Sec. V-B that change rarely (dw_config): kept in
+// the workspace for the kernels that run the rule at their end.
+struct RuleConfig {
+    double coef[AH_MAX_HIST];  // c_0 .. c_{p-1}, c_0 on the newest difference
+    double kappa;              // threshold of h1 / h2, negative
+    int p_hist;                // history depth p
+    int reserved;
+};
+
+// Where the squared distances ||x_i - c||^2 of a round are assembled.  Level 0 holds one
+// sum per (worker, tile); every higher level holds, per worker, the adjacent-pairs tree
+// sums of 64 consecutive nodes of the level below, up to a single root.  A node of level
+// L >= 1 also has an arrival counter: whoever delivers the last live child of a node sums
+// its children (in the fixed tree order, so the value does not depend on who does it),
+// resets the counter and delivers the node to its own parent.  Nobody waits for anybody.
+// The root of worker i is norm2[i]; whoever completes the last worker copies the K
+// results (and the status word) to pinned host memory and, when asked, runs the
+// weighting rule on them.  All counters are zero between rounds.
+constexpr int kTreeRadixLog2 = 6;
+constexpr int kTreeMaxLevels = 4;      // 2^21 tiles at most (P < 2^31, 1024 parameters a tile)
+struct DistTree {
+    double *level0;                    // [K][n[0]], n[0] = tiles rounded up to a power of two
+    double *upper;                     // level L >= 1: upper + K * off[L] + i * n[L] + node
+    uint32_t *count;                   // same indexing as upper
+    uint32_t *rows_done;               // workers whose root is complete this round
+    double *norm2;                     // [K] roots
+    double *norm2_host;                // pinned, mapped: [0] status word, [1 .. K] roots
+    const uint32_t *status;            // device status word
+    const RuleConfig *rule;            // the rule at the end of the round: its parameters,
+    double *uhist;                     //   the history ring [K][p + 1] on the device,
+    uint32_t *ring_flag;               //   whether the ring has been filled,
+    float *weights;                    //   and where the coefficients go: h2[K] then h1[K]
+    double rule_alpha;
+    uint32_t run_rule;                 // 1: run the rule once every root is complete
+    uint32_t K;
+    uint32_t levels;                   // level `levels` is the root (n == 1)
+    uint32_t n[kTreeMaxLevels + 1];    // nodes per worker at each level
+    uint32_t live[kTreeMaxLevels + 1]; // of which exist (the others count as +0, never read)
+    uint32_t off[kTreeMaxLevels + 1];  // nodes per worker in the levels 1 .. L-1
+};
+
+// Launch parameters of the fused local step.  The per-worker tables are sized by the
+// template argument: a launch for K <= 16 workers carries half a kilobyte of them, not
+// the 7 KB that 256 workers need.
+struct StepCommon {
     float *x, *m, *v;
     const float *c;
     const float *grad, *hvp;
-    double *partials;          // [K][ntiles_pad] tile sums of (x - c)^2
     uint32_t *status;          // device status word
     uint32_t *sched;           // [0] next item to hand out, [1] producers that have left;
                                // both zero between launches
@@ -90,16 +140,12 @@ struct StepParams {
     uint64_t ld;               // row stride of grad, hvp
     uint32_t P;
     uint32_t ntiles;
-    uint32_t ntiles_pad;       // power of two >= ntiles
     uint32_t key0, key1, round;
     float lr, beta1, beta2, omb1, omb2, eps, hpow, wd;
     uint32_t nsamp;            // Hutchinson samples per step (1 .. AH_MAX_SAMPLES)
     uint64_t sample_stride;    // elements between consecutive samples in hvp
     uint32_t nrows;            // worker rows to process (all K when distances are wanted)
     uint32_t nitems;           // nrows * ntiles
-    WorkerConst w[AH_MAX_WORKERS];
-    uint16_t row[AH_MAX_WORKERS];     // row r -> worker index
-    uint8_t active[AH_MAX_WORKERS];   // by worker index
     // fused step + exchange (one pass on exchange rounds); unused otherwise
     uint32_t fused;                   // 1: an item is a tile with all its workers, in row order
     uint32_t asynchronous;            // 1: workers meet the master one at a time, in row order
@@ -108,10 +154,21 @@ struct StepParams {
     uint32_t nworkers;                // K, for the layout of wdev
     float *c_out;                     // the master row, written once per tile
     const float *wdev;                // not null: h2 of worker i at wdev[i], h1 at wdev[K + i]
-    float h1w[AH_MAX_WORKERS];        // else the coefficients by worker index
-    float h2w[AH_MAX_WORKERS];
-    uint8_t exch[AH_MAX_WORKERS];     // by worker index: meets the master this round
+    DistTree tree;                    // distance rounds only
 };
+
+template <int MAXW>
+struct StepParamsT : StepCommon {
+    WorkerConst w[MAXW];
+    float h1w[MAXW];                  // coefficients by worker index when wdev is null
+    float h2w[MAXW];
+    uint16_t row[MAXW];               // row r -> worker index
+    uint8_t active[MAXW];             // by worker index
+    uint8_t exch[MAXW];               // by worker index: meets the master this round
+};
+constexpr int kFewWorkers = 16;
+using StepParams = StepParamsT<AH_MAX_WORKERS>;      // what the host fills in
+using StepParamsFew = StepParamsT<kFewWorkers>;      // what a launch for K <= 16 carries
 
 struct ExchangeParams {
     float *x;
@@ -143,8 +200,6 @@ __device__ __forceinline__ float exchange_h2(const ExchangeParams &p, int a)
 
 // Kernel launchers (ah_kernels.cu).  Each returns the cudaError_t of the launch.
 cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);
-cudaError_t launch_norm2_finalize(double *partials, double *scratch, uint32_t ntiles,
-                                  uint32_t ntiles_pad, int K, double *norm2, cudaStream_t s);
 cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s);
 cudaError_t launch_sample_z(float *dst, uint64_t ld, uint32_t P, int K, uint32_t key0,
                             uint32_t key1, uint32_t round, uint32_t sample, cudaStream_t s);

@@ -13,6 +13,7 @@
 
 #include "ah_internal.h"
 #include "ah_device.cuh"
+#include "ah_tree.cuh"
 
 namespace ah {
 
@@ -136,14 +137,14 @@ __device__ __forceinline__ float max_abs4(float4 a)
 // share one test of the division window.  D is the spatially averaged Hutchinson
 // estimate of the Hessian diagonal for this element.
 // POWMODE: 0 -> k = 1, 1 -> k = 1/2, 2 -> general k via powf.
-__device__ __forceinline__ void moments(float &m, float &v, float g, float D, const StepParams &p)
+__device__ __forceinline__ void moments(float &m, float &v, float g, float D, const StepCommon &p)
 {
     m = __fadd_rn(__fmul_rn(p.beta1, m), __fmul_rn(p.omb1, g));
     v = __fadd_rn(__fmul_rn(p.beta2, v), __fmul_rn(__fmul_rn(p.omb2, D), D));
 }
 
 template <int POWMODE, bool WD, bool WINDOW>
-__device__ __forceinline__ float step_from_moments(float x, float m1, float v1, const StepParams &p,
+__device__ __forceinline__ float step_from_moments(float x, float m1, float v1, const StepCommon &p,
                                                    const WorkerConst &w)
 {
     const float mhat = WINDOW ? div_by_const_in_window(m1, w.bc1, w.rbc1) : __fdiv_rn(m1, w.bc1);
@@ -161,7 +162,7 @@ __device__ __forceinline__ float step_from_moments(float x, float m1, float v1, 
 
 template <int POWMODE, bool WD>
 __device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, float g, float D,
-                                                  const StepParams &p, const WorkerConst &w)
+                                                  const StepCommon &p, const WorkerConst &w)
 {
     moments(m, v, g, D, p);
     const float lo = fminf(fabsf(m), fabsf(v)), hi = fmaxf(fabsf(m), fabsf(v));
@@ -172,7 +173,7 @@ __device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, 
 // Four consecutive elements at once: one window test for the eight divisions.
 template <int POWMODE, bool WD>
 __device__ __forceinline__ void adahessian_update4(float4 &x, float4 &m, float4 &v, const float4 g,
-                                                   const float4 D, const StepParams &p,
+                                                   const float4 D, const StepCommon &p,
                                                    const WorkerConst &w)
 {
     moments(m.x, v.x, g.x, D.x, p);
@@ -221,22 +222,32 @@ __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 //
 // Producer warp, per item: waits until the stage is free, computes the Philox
 // blocks whose bits are the Rademacher signs of the tile (one lane per group of 128
-// parameters), writes a small header, and issues bulk copies of grad, x, m, v, (c)
-// and of the Hessian-vector values of the tile widened to whole spatial blocks.  z
-// costs no memory traffic.
+// parameters), writes the item's header (everything the consumers would otherwise
+// work out per thread: which worker, its bias corrections, its exchange coefficients,
+// the tile's extent), and issues bulk copies of grad, x, m, v, (c) and of the
+// Hessian-vector values of the tile widened to whole spatial blocks.  z costs no
+// memory traffic.
 //
-// Consumers, per item: wait for the stage; where the tile touches a tensor with
-// spatial block > 1 they turn hvp into z (.) hvp in place, average each block in
-// place (one thread per block, ascending-order sum, one division) and read the
-// means back; otherwise the sign is applied in registers.  Tiles whose averaged
-// tensors are all 3 x 3 kernels (the common case) skip the separate sign pass: the
-// thread that sums a block takes the nine signs from the Philox words as it goes.
-// Then moments and update per element, 128-bit stores of x, m, v, and the stage goes
-// back to the producer.
+// Consumers, per item: wait for the stage and agree through one reducing barrier that
+// it has arrived (so that they all go on or all leave); where the tile touches a tensor
+// with spatial block > 1 they turn hvp into z (.) hvp in place, average each block in
+// place (one thread per block, ascending-order sum, one division) and read the means
+// back; otherwise the sign is applied in registers.  Tiles whose averaged tensors are
+// all 3 x 3 kernels (the common case) skip the separate sign pass: the thread that sums
+// a block takes the nine signs from the Philox words as it goes.  Then moments and
+// update per element, 128-bit stores of x, m, v, and the stage goes back to the producer.
 //
-// DIST additionally leaves, per tile, the pairwise-tree sum of (x_new - c)^2 in
-// p.partials[worker][tile], for every worker; a worker that sits the step out
-// contributes its unchanged x (only x and c are fetched for it).
+// DIST additionally forms, per item, the pairwise-tree sum of (x_new - c)^2: the
+// consumer warps leave their eight partial sums in the stage, and the producer, when it
+// takes the stage back, adds them up and delivers the tile's sum to the arrival tree of
+// ah_tree.cuh, which ends in the K distances (and, if asked, the weighting rule) without
+// a launch of its own.  A worker that sits the step out contributes its unchanged x
+// (only x and c are fetched for it).
+//
+// The kernel may be launched with programmatic stream serialisation: everything before
+// griddepcontrol.wait touches only this CTA's shared memory and the launch parameters;
+// the first draw from the item counter and every access to state, inputs and workspace
+// come after it.
 // ---------------------------------------------------------------------------
 enum : uint32_t {
     kItemAverage = 1u,        // the tile touches a spatial block > 1
@@ -248,11 +259,23 @@ enum : uint32_t {
     kItemAll3x3 = 64u,        // every averaged tensor the tile touches has block 9
 };
 
-template <bool HASC>
-struct __align__(128) Stage {
+constexpr int kRed = kPasses * kConsumerWarps;     // per-warp, per-pass sums of a tile
+static_assert((kRed & (kRed - 1)) == 0 && kRed <= 32, "the tile's sums form a subtree");
+
+// What the producer tells the consumers about an item: four 16-byte words.
+struct __align__(16) ItemHeader {
     uint32_t worker, t0, nvalid, flags;
     uint32_t e0, e1, run0, ea0;
-    uint32_t tile, reserved[7];
+    float bc1, bc2, rbc1, rbc2;            // the worker's bias corrections and reciprocals
+    uint32_t tile;
+    float h1, h2;                          // fused exchange: the worker's coefficients
+    uint32_t reserved;
+};
+
+template <bool HASC>
+struct __align__(128) Stage {
+    ItemHeader hdr;
+    double red[kRed];                      // DIST: sums of (x - c)^2, one per warp and pass
     uint32_t zw[kStageGroups][4];          // Philox words of groups (ea0 >> 7) ...
     float g[kTile], x[kTile], m[kTile], v[kTile];
     float c[HASC ? kTile : 4];
@@ -266,13 +289,34 @@ struct __align__(128) ExtraSample {
     float hv[kTile + 2 * kHalo];
 };
 
-template <bool HASC>
+template <bool HASC, bool FUSE, int MAXW>
 struct __align__(128) Shared {
     Stage<HASC> stage[kStages];
     uint64_t full[kStages];                // producer -> consumers (bytes landed)
     uint64_t empty[kStages];               // consumers -> producer (stage drained)
-    double red[2][kPasses * kConsumerWarps];
+    float h1[FUSE ? MAXW : 1];             // fused exchange: coefficients by worker index
+    float h2[FUSE ? MAXW : 1];
 };
+
+// All consumers learn whether every one of them saw the stage arrive.
+__device__ __forceinline__ bool consumers_agree(bool mine)
+{
+    uint32_t all;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "barrier.cta.red.and.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(all)
+        : "r"((uint32_t)mine), "n"(kConsumers)
+        : "memory");
+    return all != 0u;
+}
+
+__device__ __forceinline__ uint4 ld_shared_u4(const void *p)
+{
+    return *reinterpret_cast<const uint4 *>(p);
+}
 
 template <int B>
 __device__ __forceinline__ void block_means_fixed(float *base, uint32_t nblk, int ctid)
@@ -376,14 +420,80 @@ __device__ __forceinline__ float4 hutchinson4(const Stage<HASC> &st, const Extra
     return D;
 }
 
-template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
-local_step_kernel(const __grid_constant__ StepParams p)
+// By the producer warp, on a stage the consumers have handed back: the tile's sum of
+// (x - c)^2 from the per-warp, per-pass sums (top levels of the adjacent-pairs tree).
+template <bool HASC>
+__device__ __forceinline__ double stage_sum(const Stage<HASC> &st, int lane)
+{
+    double v = st.red[lane & (kRed - 1)];          // every group of kRed lanes forms the same sum
+#pragma unroll
+    for (int off = 1; off < kRed; off <<= 1)
+        v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, off));
+    return v;
+}
+
+// The producer's deliveries to the arrival tree, in batches of up to 32 so that the
+// memory round trips they need (a fence, the counters) are paid once per batch and never
+// hold up the next bulk copies.  Lane e of the producer owns entry e of a batch: it stores
+// the tile's sum at once (nobody waits for a store), and when the batch is full it fences
+// and counts its entry; what the counter returned is looked at when the next batch is
+// counted, or at the end.
+struct Deliveries {
+    uint32_t fill = 0;                      // entries of the batch being filled (same in every lane)
+    uint32_t my_i = 0, my_tile = 0;         // this lane's entry of that batch
+    uint32_t counted = 0;                   // entries of the batch whose counts are in flight
+    uint32_t c_i = 0, c_tile = 0, c_before = 0;   // this lane's entry of that batch
+
+    // the counts of the previous batch have come back: finish the nodes they completed
+    __device__ __forceinline__ void settle(const DistTree &T, int lane)
+    {
+        tree_after_counts(T, (uint32_t)lane < counted, c_i, c_tile, c_before, lane);
+        counted = 0;
+    }
+
+    // count the batch that has been filled
+    __device__ __forceinline__ void count(const DistTree &T, int lane)
+    {
+        settle(T, lane);
+        if ((uint32_t)lane < fill) c_before = tree_count_tile(T, my_i, my_tile);
+        c_i = my_i; c_tile = my_tile;
+        counted = fill;
+        fill = 0;
+    }
+
+    // a new tile sum (v in every lane)
+    __device__ __forceinline__ void add(const DistTree &T, uint32_t i, uint32_t tile, double v, int lane)
+    {
+        if ((uint32_t)lane == fill) {
+            tree_store_tile(T, i, tile, v);
+            my_i = i; my_tile = tile;
+        }
+        if (++fill == 32u) count(T, lane);
+    }
+
+    // nothing more comes: everything in flight is counted and settled
+    __device__ __forceinline__ void finish(const DistTree &T, int lane)
+    {
+        count(T, lane);
+        settle(T, lane);
+    }
+};
+
+// CTAs per SM an instantiation is built (register bound) and launched for.
+constexpr int ctas_per_sm(bool dist, bool multi, bool fuse)
+{
+    return dist || multi || fuse ? kCtasPerSm : kCtasPerSmPlain;
+}
+
+template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE, int MAXW>
+__global__ void __launch_bounds__(kThreads, ctas_per_sm(DIST, MULTI, FUSE))
+local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
 {
     constexpr bool HASC = DIST || FUSE;            // the stages carry a tile of the master row
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    Shared<HASC> &sh = *reinterpret_cast<Shared<HASC> *>(smem_raw);
-    ExtraSample *extra = reinterpret_cast<ExtraSample *>(smem_raw + sizeof(Shared<HASC>));
+    using SharedT = Shared<HASC, FUSE, MAXW>;
+    SharedT &sh = *reinterpret_cast<SharedT *>(smem_raw);
+    ExtraSample *extra = reinterpret_cast<ExtraSample *>(smem_raw + sizeof(SharedT));
     const uint32_t nextra = MULTI ? p.nsamp - 1u : 0u;     // extra samples per stage
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -395,24 +505,43 @@ local_step_kernel(const __grid_constant__ StepParams p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // a launch that was allowed to start early waits here for the launches before it
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == kConsumerWarps) {
         // =============================== producer ===============================
+        if constexpr (FUSE) {
+            // exchange coefficients by worker index, from the device-side rule or the launch
+            for (uint32_t w = (uint32_t)lane; w < p.nworkers; w += 32u) {
+                sh.h1[w] = p.wdev ? p.wdev[p.nworkers + w] : p.h1w[w];
+                sh.h2[w] = p.wdev ? p.wdev[w] : p.h2w[w];
+            }
+            __syncwarp();
+        }
         // Items are drawn from the global counter one ahead of their use, so that the
         // round trip of the atomic overlaps the wait for a free stage.
         uint32_t drawn = 0;
         if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
         uint32_t k = 0;
         uint32_t tile = 0, r = 0, rows_left = 0;   // FUSE: where the producer is in a tile's worker list
+        bool healthy = true;
+        Deliveries deliveries;                     // DIST: tile sums on their way into the tree
         for (;; ++k) {
             const uint32_t s = k % kStages, use = k / kStages;
-            if (use > 0 && !mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout))
-                break;
+            Stage<HASC> &st = sh.stage[s];
+            if (use > 0) {
+                if (!mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout)) {
+                    healthy = false;
+                    break;
+                }
+                if constexpr (DIST)                // the item that just left this stage
+                    deliveries.add(p.tree, st.hdr.worker, st.hdr.tile, stage_sum(st, lane), lane);
+            }
             if (!FUSE || rows_left == 0u) {
                 const uint32_t n = __shfl_sync(0xffffffffu, drawn, 0);
                 if (n >= p.nitems) {         // nothing left: tell the consumers and leave
                     if (lane == 0) {
-                        sh.stage[s].flags = kItemEnd;
+                        st.hdr.flags = kItemEnd;
                         mbar_arrive(&sh.full[s]);
                     }
                     break;
@@ -429,7 +558,6 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     r = DIST ? n - tile * p.nrows : n / p.ntiles;
                 }
             }
-            Stage<HASC> &st = sh.stage[s];
             const uint32_t i = p.row[r];
             const bool act = p.active[i] != 0;
             const uint32_t t0 = tile * (uint32_t)kTile;
@@ -452,13 +580,20 @@ local_step_kernel(const __grid_constant__ StepParams p)
             }
             const bool first = FUSE && r == 0u, last = FUSE && rows_left == 1u;
             if (lane == 0) {
-                st.worker = i; st.t0 = t0; st.nvalid = nvalid;
-                st.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly) |
+                ItemHeader hd;
+                hd.worker = i; hd.t0 = t0; hd.nvalid = nvalid;
+                hd.flags = (avg ? kItemAverage : 0u) | (act ? 0u : kItemDistanceOnly) |
                            ((ti.flags & 2u) ? kItemAll3x3 : 0u) |
                            (first ? kItemFirst : 0u) | (last ? kItemLast : 0u) |
                            (FUSE && p.exch[i] ? kItemExchange : 0u);
-                st.e0 = ti.e0; st.e1 = ti.e1; st.run0 = ti.run0; st.ea0 = ea0;
-                st.tile = tile;
+                hd.e0 = ti.e0; hd.e1 = ti.e1; hd.run0 = ti.run0; hd.ea0 = ea0;
+                const WorkerConst wc = p.w[i];
+                hd.bc1 = wc.bc1; hd.bc2 = wc.bc2; hd.rbc1 = wc.rbc1; hd.rbc2 = wc.rbc2;
+                hd.tile = tile;
+                hd.h1 = FUSE ? sh.h1[i] : 0.f;
+                hd.h2 = FUSE ? sh.h2[i] : 0.f;
+                hd.reserved = 0u;
+                st.hdr = hd;
             }
             __syncwarp();
             if (lane == 0) {
@@ -489,6 +624,20 @@ local_step_kernel(const __grid_constant__ StepParams p)
             }
             if constexpr (FUSE) { ++r; --rows_left; }
         }
+        // this CTA draws no more items: a launch waiting behind this one may move in as the
+        // CTAs leave (it still waits for this whole launch before it touches memory)
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        if constexpr (DIST) {
+            // the items still with the consumers, in the order in which they finish
+            for (uint32_t j = k + 1u; healthy && j < k + (uint32_t)kStages; ++j) {
+                const uint32_t s = j % kStages, use = j / kStages;
+                if (use == 0u) continue;
+                if (!mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout)) break;
+                const Stage<HASC> &st = sh.stage[s];
+                deliveries.add(p.tree, st.hdr.worker, st.hdr.tile, stage_sum(st, lane), lane);
+            }
+            deliveries.finish(p.tree, lane);
+        }
         // the last producer to leave puts both scheduler words back to zero for the next
         // launch (every producer has made its final fetch before it counts itself out)
         if (lane == 0) {
@@ -507,9 +656,12 @@ local_step_kernel(const __grid_constant__ StepParams p)
     uint32_t k = 0;
     for (;; ++k) {
         const uint32_t s = k % kStages, use = k / kStages;
-        if (!mbar_wait(&sh.full[s], use & 1u, p.status, kStatusFullTimeout)) break;
+        // every consumer polls (bounded); one reducing barrier makes the verdict common, so
+        // that nobody is left behind at a later barrier by a warp that gave up
+        if (!consumers_agree(mbar_wait(&sh.full[s], use & 1u, p.status, kStatusFullTimeout))) break;
         Stage<HASC> &st = sh.stage[s];
-        const uint32_t i = st.worker, t0 = st.t0, nvalid = st.nvalid, flags = st.flags;
+        const uint4 h0 = ld_shared_u4(&st.hdr.worker);
+        const uint32_t i = h0.x, t0 = h0.y, nvalid = h0.z, flags = h0.w;
         if (flags & kItemEnd) break;
         const ExtraSample *xs = extra + s * nextra;
         const float fn = (float)p.nsamp, rn = __frcp_rn(fn);
@@ -520,10 +672,8 @@ local_step_kernel(const __grid_constant__ StepParams p)
         const bool meets_first = meets && p.pull_first != 0u;
         float h1 = 0.f, h2 = 0.f;
         if constexpr (FUSE) {
-            h1 = p.wdev ? p.wdev[p.nworkers + i] : p.h1w[i];
-            h2 = p.wdev ? p.wdev[i] : p.h2w[i];
-        }
-        if constexpr (FUSE) {
+            h1 = st.hdr.h1;
+            h2 = st.hdr.h2;
             if (flags & kItemFirst) {
 #pragma unroll
                 for (int pass = 0; pass < kPasses; ++pass) {
@@ -539,14 +689,17 @@ local_step_kernel(const __grid_constant__ StepParams p)
         }
 
         if (!(flags & kItemDistanceOnly)) {
-            const WorkerConst w = p.w[i];
+            const float4 wcv = ld_vec(&st.hdr.bc1);
+            WorkerConst w;
+            w.bc1 = wcv.x; w.bc2 = wcv.y; w.rbc1 = wcv.z; w.rbc2 = wcv.w;
             if (flags & kItemAverage) {
-                const uint32_t ea0 = st.ea0, ea1 = (st.e1 + 3u) & ~3u, g0 = ea0 >> 7;
-                const uint32_t e0 = st.e0, e1 = st.e1;
+                const uint4 h1w = ld_shared_u4(&st.hdr.e0);
+                const uint32_t e0 = h1w.x, e1 = h1w.y, run0 = h1w.z, ea0 = h1w.w;
+                const uint32_t ea1 = (e1 + 3u) & ~3u, g0 = ea0 >> 7;
                 if (!MULTI && (flags & kItemAll3x3)) {
                     // ---- 3x3 kernels only: means from the raw values, signs on the fly;
                     // ranges of unaveraged tensors inside the tile get their signs in place
-                    for (uint32_t ri = st.run0;; ++ri) {
+                    for (uint32_t ri = run0;; ++ri) {
                         const Run rn = p.runs[ri];
                         if (rn.start >= e1) break;
                         const uint32_t qa = max(e0, rn.start), qb = min(e1, rn.end);
@@ -571,7 +724,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     }
                     consumer_sync();
                     // ---- block means in place, one thread per block
-                    for (uint32_t ri = st.run0;; ++ri) {
+                    for (uint32_t ri = run0;; ++ri) {
                         const Run rn = p.runs[ri];
                         if (rn.start >= e1) break;
                         if (rn.block > 1u) {
@@ -629,7 +782,8 @@ local_step_kernel(const __grid_constant__ StepParams p)
         }
 
         if constexpr (DIST) {
-            double *red = sh.red[k & 1u];
+            // per warp and pass: the subtree of 128 consecutive (x - c)^2; the producer adds
+            // the kRed of them up once the stage is back with it
 #pragma unroll
             for (int pass = 0; pass < kPasses; ++pass) {
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
@@ -639,19 +793,7 @@ local_step_kernel(const __grid_constant__ StepParams p)
                     d = dist4(xn[pass], FUSE ? c_old[pass] : ld_vec(&st.c[off]), nv);
                 }
                 d = warp_tree_sum(d);
-                if (lane == 0) red[pass * kConsumerWarps + warp] = d;
-            }
-            consumer_sync();
-            if (ctid == 0) {
-                constexpr int kN = kPasses * kConsumerWarps;
-                double t[kN];
-#pragma unroll
-                for (int q = 0; q < kN; ++q) t[q] = red[q];
-#pragma unroll
-                for (int len = kN; len > 1; len >>= 1)
-#pragma unroll
-                    for (int q = 0; q < len / 2; ++q) t[q] = __dadd_rn(t[2 * q], t[2 * q + 1]);
-                p.partials[(uint64_t)i * p.ntiles_pad + st.tile] = t[0];
+                if (lane == 0) st.red[pass * kConsumerWarps + warp] = d;
             }
         }
 
@@ -682,33 +824,6 @@ local_step_kernel(const __grid_constant__ StepParams p)
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.empty[s]);
     }
-}
-
-// ---------------------------------------------------------------------------
-// ||x_i - c||^2 from the tile partials: the upper levels of the same pairwise tree,
-// one CTA per worker, ping-ponging between two rows of scratch.  Tiles that do not
-// exist (index >= ntiles) count as +0.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-norm2_finalize_kernel(double *partials, double *scratch, uint32_t ntiles, uint32_t ntiles_pad,
-                      double *norm2)
-{
-    const int i = blockIdx.x;
-    double *a = partials + (uint64_t)i * ntiles_pad;
-    double *b = scratch + (uint64_t)i * ntiles_pad;
-    uint32_t live = ntiles;
-    for (uint32_t n = ntiles_pad; n > 1; n >>= 1) {
-        const uint32_t half = n >> 1;
-        for (uint32_t k = threadIdx.x; k < half; k += blockDim.x) {
-            const double l = 2 * k < live ? a[2 * k] : 0.0;
-            const double r = 2 * k + 1 < live ? a[2 * k + 1] : 0.0;
-            b[k] = __dadd_rn(l, r);
-        }
-        __syncthreads();
-        double *t = a; a = b; b = t;
-        live = half;
-    }
-    if (threadIdx.x == 0) norm2[i] = a[0];
 }
 
 // ---------------------------------------------------------------------------
@@ -787,12 +902,13 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE>
-static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream_t s)
+template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE, int MAXW>
+static cudaError_t launch_step_one(const StepParamsT<MAXW> &p, int sm_count, cudaStream_t s)
 {
-    auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI, FUSE>;
+    auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI, FUSE, MAXW>;
     constexpr bool HASC = DIST || FUSE;
-    const size_t smem = sizeof(Shared<HASC>) +
+    using SharedT = Shared<HASC, FUSE, MAXW>;
+    const size_t smem = sizeof(SharedT) +
                         (MULTI ? (size_t)kStages * (p.nsamp - 1u) * sizeof(ExtraSample) : 0);
     // Shared-memory attributes are per device and per instantiation: one bit per device
     // ordinal.  Setting them twice is harmless, so racing threads need no lock.
@@ -802,7 +918,7 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
     if (cudaError_t e = cudaGetDevice(&device); e != cudaSuccess) return e;
     const uint64_t device_bit = 1ull << (device & 63);
     if (!(configured.load(std::memory_order_acquire) & device_bit)) {
-        const size_t most = sizeof(Shared<HASC>) +
+        const size_t most = sizeof(SharedT) +
                             (MULTI ? (size_t)kStages * (AH_MAX_SAMPLES - 1) * sizeof(ExtraSample) : 0);
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)most);
@@ -813,58 +929,79 @@ static cudaError_t launch_step_one(const StepParams &p, int sm_count, cudaStream
         configured.fetch_or(device_bit, std::memory_order_release);
     }
     if (p.nitems == 0) return cudaSuccess;
-    int ctas = kCtasPerSm;
-    if (MULTI) {                         // the extra samples decide how many CTAs fit
-        if (ctas_for_nsamp[p.nsamp].load(std::memory_order_relaxed) == 0) {
-            int fit = 0;
-            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, kThreads, smem);
-            if (e != cudaSuccess) return e;
-            if (fit < 1) return cudaErrorInvalidConfiguration;
-            ctas_for_nsamp[p.nsamp].store(fit, std::memory_order_relaxed);
-        }
-        ctas = ctas_for_nsamp[p.nsamp].load(std::memory_order_relaxed);
+    // resident CTAs per SM of this instantiation (the extra samples take shared memory)
+    const uint32_t slot = MULTI ? p.nsamp : 1u;
+    if (ctas_for_nsamp[slot].load(std::memory_order_relaxed) == 0) {
+        int fit = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, kThreads, smem);
+        if (e != cudaSuccess) return e;
+        if (fit < 1) return cudaErrorInvalidConfiguration;
+        constexpr int want = ctas_per_sm(DIST, MULTI, FUSE);
+        ctas_for_nsamp[slot].store(fit < want ? fit : want, std::memory_order_relaxed);
     }
+    const int ctas = ctas_for_nsamp[slot].load(std::memory_order_relaxed);
     const uint32_t resident = (uint32_t)sm_count * (uint32_t)ctas;
     const uint32_t grid = p.nitems < resident ? p.nitems : resident;
-    kernel<<<grid, kThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    // Programmatic stream serialisation: this launch may begin (set up its barriers, read
+    // its parameters) while the kernel before it in the stream drains; it waits for that
+    // kernel at griddepcontrol.wait before it touches memory.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
-template <int POWMODE, bool WD>
-static cudaError_t launch_step_dist(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
+template <int POWMODE, bool WD, int MAXW>
+static cudaError_t launch_step_dist(const StepParamsT<MAXW> &p, bool want_dist, int sm_count,
+                                    cudaStream_t s)
 {
     if (p.fused && p.nsamp > 1u)         // step and exchange in one pass, several samples
-        return want_dist ? launch_step_one<POWMODE, WD, true, true, true>(p, sm_count, s)
-                         : launch_step_one<POWMODE, WD, false, true, true>(p, sm_count, s);
+        return want_dist ? launch_step_one<POWMODE, WD, true, true, true, MAXW>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, true, true, MAXW>(p, sm_count, s);
     if (p.fused)                         // step and exchange in one pass
-        return want_dist ? launch_step_one<POWMODE, WD, true, false, true>(p, sm_count, s)
-                         : launch_step_one<POWMODE, WD, false, false, true>(p, sm_count, s);
+        return want_dist ? launch_step_one<POWMODE, WD, true, false, true, MAXW>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, false, true, MAXW>(p, sm_count, s);
     if (p.nsamp > 1u)
-        return want_dist ? launch_step_one<POWMODE, WD, true, true, false>(p, sm_count, s)
-                         : launch_step_one<POWMODE, WD, false, true, false>(p, sm_count, s);
-    return want_dist ? launch_step_one<POWMODE, WD, true, false, false>(p, sm_count, s)
-                     : launch_step_one<POWMODE, WD, false, false, false>(p, sm_count, s);
+        return want_dist ? launch_step_one<POWMODE, WD, true, true, false, MAXW>(p, sm_count, s)
+                         : launch_step_one<POWMODE, WD, false, true, false, MAXW>(p, sm_count, s);
+    return want_dist ? launch_step_one<POWMODE, WD, true, false, false, MAXW>(p, sm_count, s)
+                     : launch_step_one<POWMODE, WD, false, false, false, MAXW>(p, sm_count, s);
 }
 
-cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
+template <int MAXW>
+static cudaError_t launch_step_mode(const StepParamsT<MAXW> &p, bool want_dist, int sm_count,
+                                    cudaStream_t s)
 {
     const int mode = p.hpow == 1.0f ? 0 : (p.hpow == 0.5f ? 1 : 2);
     const bool wd = p.wd != 0.0f;
     switch (mode * 2 + (wd ? 1 : 0)) {
-    case 0: return launch_step_dist<0, false>(p, want_dist, sm_count, s);
-    case 1: return launch_step_dist<0, true>(p, want_dist, sm_count, s);
-    case 2: return launch_step_dist<1, false>(p, want_dist, sm_count, s);
-    case 3: return launch_step_dist<1, true>(p, want_dist, sm_count, s);
-    case 4: return launch_step_dist<2, false>(p, want_dist, sm_count, s);
-    default: return launch_step_dist<2, true>(p, want_dist, sm_count, s);
+    case 0: return launch_step_dist<0, false, MAXW>(p, want_dist, sm_count, s);
+    case 1: return launch_step_dist<0, true, MAXW>(p, want_dist, sm_count, s);
+    case 2: return launch_step_dist<1, false, MAXW>(p, want_dist, sm_count, s);
+    case 3: return launch_step_dist<1, true, MAXW>(p, want_dist, sm_count, s);
+    case 4: return launch_step_dist<2, false, MAXW>(p, want_dist, sm_count, s);
+    default: return launch_step_dist<2, true, MAXW>(p, want_dist, sm_count, s);
     }
 }
 
-cudaError_t launch_norm2_finalize(double *partials, double *scratch, uint32_t ntiles,
-                                  uint32_t ntiles_pad, int K, double *norm2, cudaStream_t s)
+cudaError_t launch_local_step(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s)
 {
-    norm2_finalize_kernel<<<K, 1024, 0, s>>>(partials, scratch, ntiles, ntiles_pad, norm2);
-    return cudaGetLastError();
+    if (p.nworkers > (uint32_t)kFewWorkers) return launch_step_mode(p, want_dist, sm_count, s);
+    // few workers: the launch carries per-worker tables of kFewWorkers entries
+    StepParamsFew q;
+    static_cast<StepCommon &>(q) = static_cast<const StepCommon &>(p);
+    for (int i = 0; i < kFewWorkers; ++i) {
+        q.w[i] = p.w[i]; q.h1w[i] = p.h1w[i]; q.h2w[i] = p.h2w[i];
+        q.row[i] = p.row[i]; q.active[i] = p.active[i]; q.exch[i] = p.exch[i];
+    }
+    return launch_step_mode(q, want_dist, sm_count, s);
 }
 
 cudaError_t launch_exchange(const ExchangeParams &p, cudaStream_t s)

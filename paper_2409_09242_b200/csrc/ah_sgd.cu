@@ -8,8 +8,11 @@
 // write x), 20 with it (the velocity is read and written too).  One CTA of 256
 // threads covers kTilesPerCta consecutive tiles of 1024 parameters of one worker,
 // one float4 per thread and tile, all loads issued before the first use.
+#include <string.h>
+
 #include "ah_ctx.h"
 #include "ah_device.cuh"
+#include "ah_tree.cuh"
 
 namespace ah {
 
@@ -25,9 +28,9 @@ struct SgdParams {
     float *x, *u;                  // u: velocity (the handle's first-moment rows)
     const float *c;
     const float *grad;
-    double *partials;              // [K][ntiles_pad]
+    DistTree tree;                 // DIST: where the tile sums of (x - c)^2 go
     uint64_t lds, ld;
-    uint32_t P, ntiles, ntiles_pad;
+    uint32_t P, ntiles;
     float lr, momentum;
     uint32_t nrows;
     uint16_t row[AH_MAX_WORKERS];
@@ -89,8 +92,17 @@ sgd_step_kernel(const __grid_constant__ SgdParams p)
     }
     if (DIST) {
         __syncthreads();
-        if (threadIdx.x < kTilesPerCta && tile0 + threadIdx.x < p.ntiles)
-            p.partials[(uint64_t)i * p.ntiles_pad + tile0 + threadIdx.x] = tree8(red[threadIdx.x]);
+        if (warp == 0) {
+            // one warp delivers the CTA's tile sums to the arrival tree: lane k stores and
+            // counts tile k, then every lane whose count completed a node climbs with it
+            const bool mine = lane < kTilesPerCta && tile0 + lane < p.ntiles;
+            uint32_t before = 0;
+            if (mine) {
+                tree_store_tile(p.tree, i, tile0 + lane, tree8(red[lane]));
+                before = tree_count_tile(p.tree, i, tile0 + lane);
+            }
+            tree_after_counts(p.tree, mine, i, tile0 + lane, before, lane);
+        }
     }
 }
 
@@ -205,13 +217,14 @@ exchange_then_sgd_kernel(const __grid_constant__ SgdExchangeParams p)
 // only read): the same streaming kernel with every listed row inactive.  Used by the
 // AdaHessian distance rounds so that stragglers do not travel through the local-step
 // pipeline one nearly empty item at a time.
-cudaError_t ah::launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows)
+cudaError_t ah::launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows,
+                                     const DistTree &tree)
 {
     SgdParams p;
     p.x = h->x; p.u = h->m; p.c = h->c; p.grad = nullptr;
-    p.partials = h->partials;
+    p.tree = tree;
     p.lds = h->lds; p.ld = 0;
-    p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
+    p.P = h->P; p.ntiles = h->ntiles;
     p.lr = 0.f; p.momentum = 0.f;
     p.nrows = nrows;
     for (int i = 0; i < h->K; ++i) p.active[i] = 0;
@@ -228,26 +241,34 @@ extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const s
     if (!(hy->momentum >= 0.f && hy->momentum < 1.f)) return AH_ERR_INVALID_ARG;
     if ((ld & 3u) != 0 || ((uintptr_t)grad & 15u) != 0) return AH_ERR_ALIGN;
 
+    if (hy->want_dist != AH_DIST_NONE && hy->want_dist != AH_DIST) return AH_ERR_INVALID_ARG;
     const bool dist = hy->want_dist != 0;
     SgdParams p;
     p.x = h->x; p.u = h->m; p.c = h->c; p.grad = grad;
-    p.partials = h->partials;
     p.lds = h->lds; p.ld = ld;
-    p.P = h->P; p.ntiles = h->ntiles; p.ntiles_pad = h->ntiles_pad;
+    p.P = h->P; p.ntiles = h->ntiles;
     p.lr = hy->lr; p.momentum = hy->momentum;
     p.nrows = 0;
+    uint32_t step[AH_MAX_WORKERS];                // step counts once the launch is enqueued
     for (int i = 0; i < h->K; ++i) {
         const bool on = !hy->active || hy->active[i] != 0;
         p.active[i] = on ? 1 : 0;
-        if (on) h->step[i] += 1;
+        step[i] = h->step[i] + (on ? 1u : 0u);
         if (on || dist) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
     }
-    h->calls += 1;
+    if (dist) {
+        const int rc = prepare_distance_round(h, false, 0.f, p.tree);
+        if (rc != AH_OK) return rc;
+    } else {
+        memset(&p.tree, 0, sizeof p.tree);
+    }
     cudaError_t e;
     const bool mom = hy->momentum != 0.f;
     if (mom) e = dist ? launch_sgd<true, true>(p, h->stream) : launch_sgd<true, false>(p, h->stream);
     else     e = dist ? launch_sgd<false, true>(p, h->stream) : launch_sgd<false, false>(p, h->stream);
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->calls += 1;
+    memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
     if (p.nrows) h->launches += 1;
     if (dist) return finish_distances(h);
     return AH_OK;
@@ -278,6 +299,7 @@ extern "C" int easgd_exchange_then_sgd_step(ah_ctx *h, const float *grad, uint64
     p.asynchronous = asynchronous ? 1u : 0u;
     p.any_exchange = 0u;
     p.nrows = 0;
+    uint32_t step[AH_MAX_WORKERS];                // step counts once the launch is enqueued
     for (int q = 0; q < h->K; ++q) {
         const int i = asynchronous && order ? (int)order[q] : q;
         const bool on = !hy->active || hy->active[i] != 0;
@@ -287,16 +309,20 @@ extern "C" int easgd_exchange_then_sgd_step(ah_ctx *h, const float *grad, uint64
         if (meets) p.any_exchange = 1u;
         p.h2w[i] = weights ? weights[i] : alpha;
         p.h1w[i] = weights ? weights[h->K + i] : alpha;
-        if (on) h->step[i] += 1;
+        step[i] = h->step[i] + (on ? 1u : 0u);
         if (on || meets) p.row[p.nrows++] = (uint16_t)i;
     }
-    h->calls += 1;
-    if (p.nrows == 0) return AH_OK;
+    if (p.nrows == 0) {
+        h->calls += 1;
+        return AH_OK;
+    }
     const unsigned blocks = (p.nvec + 255u) / 256u;
     if (hy->momentum != 0.f) exchange_then_sgd_kernel<true><<<blocks, 256, 0, h->stream>>>(p);
     else                     exchange_then_sgd_kernel<false><<<blocks, 256, 0, h->stream>>>(p);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
+    h->calls += 1;
+    memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
     h->launches += 1;
     return AH_OK;
 }

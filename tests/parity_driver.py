@@ -96,8 +96,14 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                 pending = None
                 assert not ex, "tau >= 2"
             else:
+                # every other distance round also runs the weighting rule in its last kernel
+                # (AH_DIST_AND_RULE, the shape the benchmark times); the others leave it to
+                # the call that makes the exchange
+                rule_now = ex and cfg.dynamic and log["exchanges"] % 2 == 0
                 h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
-                                active=mask_g if cfg.frozen else None, **common)
+                                active=mask_g if cfg.frozen else None,
+                                **dict(common, want_dist=binding.AH_DIST_AND_RULE if rule_now else ex,
+                                       rule_alpha=alpha))
             ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
                            active=mask_o if cfg.frozen else None, **common)
             if ex:
@@ -150,9 +156,17 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                 log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], lagged_weights[0]) and
                                              np.array_equal(w[cfg.K:], lagged_weights[1]))
             continue
+        # where the weights of this exchange come from: the device (the rule either in the
+        # last kernel of the distance round or as a launch of its own) or the host
+        ex_index = log["exchanges"] + 1
+        on_device = ex and cfg.dynamic and (cfg.sync_free == "yes" or
+                                            (cfg.sync_free == "mixed" and ex_index % 2 == 1))
+        rule_now = on_device and ex_index % 3 != 0
         if cfg.method == "adahessian":
             h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
-                            active=mask_g if cfg.frozen else None, **common)
+                            active=mask_g if cfg.frozen else None,
+                            **dict(common, want_dist=binding.AH_DIST_AND_RULE if rule_now else ex,
+                                   rule_alpha=alpha))
             ref.local_step(pool[k][0], pool[k][1], Z_SEED, t,
                            active=mask_o if cfg.frozen else None, **common)
         else:
@@ -164,8 +178,6 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
         if ex:
             log["exchanges"] += 1
             w = h2 = h1 = None
-            on_device = cfg.dynamic and (cfg.sync_free == "yes" or
-                                         (cfg.sync_free == "mixed" and log["exchanges"] % 2 == 1))
             order_g = order_o = None
             if cfg.asynchronous:
                 order_g = h.dw_order_next(ORDER_SEED, t)

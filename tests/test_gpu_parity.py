@@ -901,6 +901,104 @@ def test_checkpoint_resume_with_the_rule_on_the_device(B, torch):
     h_b.close()
 
 
+def test_checkpoint_resume_with_an_exchange_pending(B, torch):
+    # the bench's default shape: the exchange of a period rides on the first local step of the
+    # next one, so at a period boundary something waits on the device: the distances (the rule
+    # still to run), or the coefficients the rule made of them at the end of the distance
+    # round.  A snapshot taken there, restored into a fresh handle, must continue bit for bit:
+    # in the first case the restored distances are pending again, in the second the restored
+    # coefficients are handed to the exchange as caller weights.
+    layout = W.resnet18_layout(16)
+    segs, P, K, tau = W.segments(layout), W.total_params(layout), 4, 2
+    theta0, pool = _layout_inputs(layout, K)
+    dev_pool = [(torch.from_numpy(g).cuda(), torch.from_numpy(hv).cuda()) for g, hv in pool]
+    from parity_driver import MASK_SEED
+
+    def rounds(h, first, last, pending, rule_in_round, restored_weights=None):
+        for t in range(first, last + 1):
+            mask = h.dw_mask_next(MASK_SEED, t, 0.2)
+            g, hv = dev_pool[t % len(dev_pool)]
+            if pending is not None:
+                if restored_weights is not None:
+                    h.easgd_exchange_then_step(g, hv, Z_SEED, lr=0.01, round_=t, worker_mask=pending,
+                                               weights=restored_weights, dynamic=False)
+                    restored_weights = None
+                else:
+                    h.easgd_exchange_then_step(g, hv, Z_SEED, lr=0.01, round_=t, worker_mask=pending,
+                                               alpha=0.05, dynamic=True)
+                pending = None
+            else:
+                ex = t % tau == 0
+                h.ah_local_step(g, hv, Z_SEED, lr=0.01, round_=t, rule_alpha=0.05,
+                                want_dist=(B.AH_DIST_AND_RULE if rule_in_round else B.AH_DIST) if ex else 0)
+                if ex:
+                    pending = mask
+        return pending
+
+    def fresh():
+        h = B.Handle(K, P, segs)
+        h.ah_state_set(B.AH_CENTER, theta0)
+        h.ah_broadcast_center()
+        return h
+
+    for rule_in_round in (False, True):
+        h_full = fresh()
+        rounds(h_full, 1, 20, None, rule_in_round)
+        h_a = fresh()
+        pending = rounds(h_a, 1, 10, None, rule_in_round)          # round 10 measured distances
+        assert pending is not None
+        sel = [B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER, B.AH_STEP, B.AH_UHIST, B.AH_DOWN_UNTIL, B.AH_ROUND]
+        sel.append(B.AH_WEIGHTS if rule_in_round else B.AH_NORM2)
+        snap = {w: h_a.ah_state_get(w) for w in sel}
+        h_a.close()
+        h_b = B.Handle(K, P, segs)
+        for w, val in snap.items():
+            h_b.ah_state_set(w, val)
+        rounds(h_b, 11, 20, pending, rule_in_round, snap[B.AH_WEIGHTS] if rule_in_round else None)
+        for w in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER, B.AH_WEIGHTS):
+            a, b = h_full.ah_state_get(w), h_b.ah_state_get(w)
+            assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), (rule_in_round, w)
+        assert np.array_equal(h_full.ah_state_get(B.AH_UHIST), h_b.ah_state_get(B.AH_UHIST))
+        h_full.close()
+        h_b.close()
+
+
+def test_library_log_distance_on_the_device(B, torch):
+    # u = log ||x_i - c|| as the device forms of the rule compute it (the rule as a launch of
+    # its own, and the rule at the end of a distance round), against the definition in
+    # 300-bit arithmetic: the natural logarithm rounded to the nearest double, halved
+    import mpmath
+    mpmath.mp.prec = 300
+    rng = np.random.default_rng(78)
+    K, P = 64, 2048
+    n2 = np.concatenate([np.exp(rng.uniform(-680, 700, 4 * K)), rng.uniform(0.5, 2.0, 3 * K),
+                         1.0 + rng.uniform(-1, 1, K) * 1e-9, np.exp(2 * rng.normal(0, 3, 4 * K))])
+    h = B.Handle(K, P, [])
+    h.dw_config(1, np.array([1.0]), -0.1)
+    for lo in range(0, n2.size, K):
+        chunk = n2[lo:lo + K]
+        h.ah_state_set(B.AH_NORM2, chunk)                  # restored distances are pending
+        h.easgd_exchange_dynamic(np.zeros(K, np.uint8), 0.05, None, False)   # the rule; nobody arrives
+        u = h.ah_state_get(B.AH_UHIST, p_hist=1)[:, 0]
+        want = np.array([float(mpmath.log(mpmath.mpf(float(v)))) * 0.5 for v in chunk])
+        assert np.array_equal(u, want), (lo, chunk[u != want][:3])
+    # the rule at the end of a distance round: x = c + d e_0 gives ||x_i - c||^2 = d_i^2 exactly
+    d = np.exp(rng.uniform(-20, 20, K)).astype(np.float32)
+    x = np.zeros((K, P), np.float32)
+    x[:, 0] = d
+    h.ah_state_set(B.AH_CENTER, np.zeros(P, np.float32))
+    h.ah_state_set(B.AH_X, x)
+    z = torch.zeros((K, P), device="cuda")
+    h.ah_local_step(z, z, 1, lr=0.0, active=np.zeros(K, np.uint8), want_dist=B.AH_DIST_AND_RULE,
+                    rule_alpha=0.05)
+    u = h.ah_state_get(B.AH_UHIST, p_hist=1)[:, 0]
+    n2d = d.astype(np.float64) ** 2
+    assert np.array_equal(h.ah_state_get(B.AH_NORM2), n2d)
+    want = np.array([float(mpmath.log(mpmath.mpf(float(v)))) * 0.5 for v in n2d])
+    assert np.array_equal(u, want)
+    h.close()
+
+
 def test_error_paths_and_own_allocation(B, torch):
     K, P = 2, 1000
     h = B.Handle(K, P, [], own_alloc=True)           # cudaMalloc workspace, default stream
@@ -922,7 +1020,20 @@ def test_error_paths_and_own_allocation(B, torch):
     # the handle still works after the refusals
     h.ah_local_step(g, g, 1, lr=0.01, want_dist=True)
     assert np.all(h.dw_weights_next(0.1) == np.float32(0.1))
-    assert h.ah_launch_count() == 2
+    assert h.ah_launch_count() == 1                  # the distances cost no launch of their own
+    # a refused call changes nothing: step counts and the call counter stay where they were
+    steps, calls = h.ah_state_get(B.AH_STEP).copy(), h.ah_state_get(B.AH_ROUND).copy()
+    assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 1002, 1, C.byref(hy)) == B.AH_ERR_ALIGN
+    far = B.ah_hyper(0.01, 0.9, 0.999, 1e-4, 1.0, 0.0, 1, None, 3)       # want_dist out of range
+    assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 1004, 1, C.byref(far)) == B.AH_ERR_INVALID_ARG
+    order = (C.c_uint16 * K)(0, 0)                                       # names worker 0 twice
+    assert lib.ah_local_step_exchange(h._h, g.data_ptr(), g.data_ptr(), 1004, 1, C.byref(hy), None, None,
+                                      0.1, order, 1, 0) == B.AH_ERR_INVALID_ARG
+    assert lib.easgd_exchange_then_step(h._h, g.data_ptr(), g.data_ptr(), 1004, 1, C.byref(hy), None, None,
+                                        0.1, None, 0, 1) == B.AH_ERR_STATE  # no distances pending
+    assert np.array_equal(h.ah_state_get(B.AH_STEP), steps)
+    assert np.array_equal(h.ah_state_get(B.AH_ROUND), calls)
+    assert h.ah_launch_count() == 1
     h.close()
     # a workspace that is too small is refused
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")

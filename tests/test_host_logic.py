@@ -73,6 +73,42 @@ def test_bookkeeping_handle_refuses_device_calls(B):
     h.close()
 
 
+def test_refused_calls_leave_the_bookkeeping_untouched(B):
+    # step counts, the call counter and the pending-distance state move only with a launch
+    # that went in: a call that is refused (here: no device behind the handle, bad arguments)
+    # leaves them exactly as they were
+    K = 3
+    h = B.Handle(K, 64, [(0, 64, 1)], host_only=True)
+    lib = B.raw()
+    steps0 = np.array([5, 0, 7], np.uint32)
+    h.ah_state_set(B.AH_STEP, steps0)
+    h.ah_state_set(B.AH_ROUND, np.array([9, 1], np.uint32))
+    hy = B.ah_hyper(0.01, 0.9, 0.999, 1e-4, 1.0, 0.0, B.AH_ROUND_AUTO, None, 1)
+    sg = B.sgd_hyper(0.01, 0.5, None, 0)
+    fake = 0x1000                                   # never dereferenced: the calls are refused first
+    order = (C.c_uint16 * K)(0, 1, 2)
+    calls = [
+        lambda: lib.ah_local_step(h._h, fake, fake, 64, 1, C.byref(hy)),
+        lambda: lib.ah_local_step(h._h, None, fake, 64, 1, C.byref(hy)),
+        lambda: lib.ah_local_step(h._h, fake, fake, 60, 1, C.byref(hy)),
+        lambda: lib.ah_local_step_exchange(h._h, fake, fake, 64, 1, C.byref(hy), None, None, 0.1, order, 1, 0),
+        lambda: lib.easgd_exchange_then_step(h._h, fake, fake, 64, 1, C.byref(hy), None, None, 0.1, None, 0, 0),
+        lambda: lib.sgd_local_step(h._h, fake, 64, C.byref(sg)),
+        lambda: lib.easgd_exchange_then_sgd_step(h._h, fake, 64, C.byref(sg), None, None, 0.1, None, 0),
+        lambda: lib.easgd_exchange_dynamic(h._h, None, 0.1, None, 0),
+        lambda: lib.ah_broadcast_center(h._h),
+    ]
+    for k, call in enumerate(calls):
+        assert call() in (B.AH_ERR_STATE, B.AH_ERR_INVALID_ARG), k
+        assert np.array_equal(h.ah_state_get(B.AH_STEP), steps0), k
+        assert list(h.ah_state_get(B.AH_ROUND)) == [9, 1], k
+        assert h.ah_launch_count() == 0
+    # the host-side rule still runs after all the refusals, from the restored history flag
+    w = h.dw_weights_from_norm2(np.array([1.0, 4.0, 9.0]), 0.05)
+    assert w.shape == (2 * K,)
+    h.close()
+
+
 def test_mask_matches_oracle_bit_for_bit(B):
     for K, p, stale in ((4, 0.1, 1), (16, 0.2, 8), (64, 0.3, 1), (8, 1 / 3, 4), (3, 0.0, 1), (3, 1.0, 2)):
         h = B.Handle(K, 8, [], host_only=True)
@@ -206,3 +242,19 @@ def test_constant_divisor_shortcut_is_exact(tmp_path):
     assert out.returncode == 0, out.stdout
     checked, bad = (int(v) for v in out.stdout.split()[1::2])
     assert checked > 200 and bad == 0
+
+
+def test_logarithm_constants_match_their_formula(tmp_path):
+    # the series coefficients 1/3 ... 1/43 of the library's logarithm are written out as pairs
+    # of doubles; a host program recomputes each from its defining formula
+    import subprocess
+    here = os.path.dirname(os.path.abspath(__file__))
+    src = os.path.join(here, "helpers", "ln_table_check.cpp")
+    csrc = os.path.join(os.path.dirname(here), "paper_2409_09242_b200", "csrc")
+    cuda_inc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "include")
+    exe = str(tmp_path / "ln_table_check")
+    subprocess.check_call(["g++", "-O1", "-std=c++17", "-ffp-contract=off", "-I", csrc, "-I", cuda_inc,
+                           src, "-o", exe])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout
+    assert out.stdout.strip().endswith("bad 0")
