@@ -67,7 +67,7 @@ NCU_TRAFFIC = {"sources_sha256": "72242c93ea8219879872e4400e4993ef0ebc408bd68804
 
 def kernel_sources_hash() -> str:
     h = hashlib.sha256()
-    for fn in ("ah_kernels.cu", "ah_internal.h", "ah_device.cuh"):
+    for fn in ("ah_local_step.cuh", "ah_step_inst.cu", "ah_tree.cuh", "ah_internal.h", "ah_device.cuh"):
         with open(os.path.join(ROOT, "paper_2409_09242_b200", "csrc", fn), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
