@@ -398,6 +398,25 @@ int dw_order_next(ah_ctx *h, uint64_t seed, uint32_t round, uint16_t *order);
 int easgd_exchange_async(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                          const uint16_t *order);
 
+/* ---- diagnostics of the arithmetic --------------------------------------------- */
+
+/* (No counterpart in the paper: a check of the implementation's own premises.)
+ * Inside its usual operand range the local step (Eq. 4: the division by (sqrt vhat)^k + eps,
+ * the square root) uses branch-free sequences in place of the general IEEE square root and
+ * division: a hardware approximation, one Newton step, a fused multiply-add on the exact
+ * residual.  They give the correctly rounded result if the refined reciprocal is the
+ * correctly rounded one (Markstein's division) and the square-root sequence rounds
+ * correctly for every input; both depend on the hardware's approximations, so this call
+ * checks them on the current device against the IEEE routines:
+ *   mismatches[0]  square root, every binary32 value in [2^-64, 2^90)
+ *   mismatches[1]  refined reciprocal, every binary32 value in [2^-33, 2^46)
+ *   mismatches[2]  quotient, division_pairs seeded pairs with |a| in [2^-63, 2^88),
+ *                  b in [2^-33, 2^46), a quarter of them with divisors next to a power of
+ *                  two, a quarter with quotients next to short significands
+ * All three must be 0.  mismatches: host pointer, 3 entries.  Synchronises; about a second
+ * for 2^32 pairs.  Makes one small cudaMalloc.  Errors: INVALID_ARG, ALLOC, CUDA. */
+int ah_check_exact_arithmetic(uint64_t division_pairs, uint64_t *mismatches, void *cuda_stream);
+
 /* ---- without a handle, without allocating ------------------------------------ */
 
 /* (No counterpart in the paper: a deployment convenience.)

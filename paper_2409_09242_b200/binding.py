@@ -37,7 +37,7 @@ EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_st
            "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step",
            "ah_local_step_exchange", "easgd_exchange_then_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "easgd_exchange_then_sgd_step", "dw_partition", "ah_distances_static", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "easgd_exchange_then_sgd_step", "dw_partition", "ah_distances_static", "ah_check_exact_arithmetic", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -96,6 +96,7 @@ _lib.easgd_exchange_async.argtypes = [_vp, C.POINTER(C.c_uint8), C.POINTER(C.c_f
 _lib.easgd_exchange_dynamic.argtypes = [_vp, C.POINTER(C.c_uint8), C.c_float, C.POINTER(C.c_uint16),
                                         C.c_int]
 _lib.ah_distances_static.argtypes = [_vp, C.c_uint64, _vp, C.c_int, C.c_uint64, _vp, _vp]
+_lib.ah_check_exact_arithmetic.argtypes = [C.c_uint64, C.POINTER(C.c_uint64), _vp]
 _lib.ah_status_string.argtypes = [C.c_int]
 _lib.ah_status_string.restype = C.c_char_p
 _lib.ah_last_cuda_error.argtypes = [_vp]
@@ -153,6 +154,19 @@ def ah_distances_static(x, c, norm2_out, stream=None):
     if rc != AH_OK:
         raise AdaHessError(rc, "ah_distances_static")
     return norm2_out
+
+
+def ah_check_exact_arithmetic(division_pairs=1 << 32, stream=None):
+    """Mismatch counts (square root, refined reciprocal, quotient) of the kernels' branch-free
+    exact routines against the IEEE routines on the current device; all must be zero."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    out = (C.c_uint64 * 3)()
+    rc = _lib.ah_check_exact_arithmetic(int(division_pairs), out, stream)
+    if rc != AH_OK:
+        raise AdaHessError(rc, "ah_check_exact_arithmetic")
+    return [int(v) for v in out]
 
 
 def dw_partition(seed, n, k, shared):

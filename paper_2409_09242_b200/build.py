@@ -18,7 +18,7 @@ _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 # compiled with different tile constants); by default the in-tree build is used.
 LIB_PATH = os.environ.get("ADAHESS_LIB") or os.path.join(_PKG, "libadahess.so")
 SOURCES = ["ah_kernels.cu", "ah_host.cu", "ah_noalloc.cu", "ah_exchange_async.cu", "ah_sgd.cu",
-           "ah_partition.cu", "ah_dynamic.cu"]
+           "ah_partition.cu", "ah_dynamic.cu", "ah_selftest.cu"]
 STEP_INSTANCES = 6          # ah_step_inst.cu, compiled with -DAH_STEP_INST=0 .. 5
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-ffp-contract=off"]

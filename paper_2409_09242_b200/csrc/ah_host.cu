@@ -525,6 +525,11 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         w.rbc2 = 1.0f / w.bc2;
     }
     p.nitems = fx ? (p.nrows ? h->ntiles : 0u) : p.nrows * h->ntiles;
+    // the branch-free exact square root and division of the kernels hold for eps in
+    // [0, 2^40] and bias corrections of at least 2^-24 (beta <= 1 - 2^-24 gives that)
+    p.narrow_ok = hy->eps >= 0.f && hy->eps <= 0x1p40f ? 1u : 0u;
+    for (int i = 0; i < h->K; ++i)
+        if (!(p.w[i].bc1 >= 0x1p-24f && p.w[i].bc2 >= 0x1p-24f)) p.narrow_ok = 0u;
 
     // ---- enqueue; the handle's bookkeeping follows each launch that went in
     if (fx && fx->dynamic && !h->rule_fresh) {

@@ -148,6 +148,8 @@ struct StepCommon {
     uint32_t ntiles;
     uint32_t key0, key1, round;
     float lr, beta1, beta2, omb1, omb2, eps, hpow, wd;
+    uint32_t narrow_ok;        // 1: eps and the bias corrections are where the branch-free exact
+                               // square root and division may be used inside the division window
     uint32_t nsamp;            // Hutchinson samples per step (1 .. AH_MAX_SAMPLES)
     uint64_t sample_stride;    // elements between consecutive samples in hvp
     uint32_t nrows;            // worker rows to process (all K when distances are wanted)

@@ -152,15 +152,18 @@ template <int POWMODE, bool WD, bool WINDOW>
 __device__ __forceinline__ float step_from_moments(float x, float m1, float v1, const StepCommon &p,
                                                    const WorkerConst &w)
 {
+    // Inside the window (and with eps in [0, 2^40], which the host checks once per launch):
+    // |mhat| in [2^-63, 2^88), vhat in [2^-63, 2^88), sqrt vhat in [2^-32, 2^44], the
+    // denominator in [2^-32, 2^45): the ranges of the branch-free exact routines.
     const float mhat = WINDOW ? div_by_const_in_window(m1, w.bc1, w.rbc1) : __fdiv_rn(m1, w.bc1);
     const float vhat = WINDOW ? div_by_const_in_window(v1, w.bc2, w.rbc2) : __fdiv_rn(v1, w.bc2);
-    const float r = __fsqrt_rn(vhat);
+    const float r = WINDOW ? sqrt_in_range(vhat) : __fsqrt_rn(vhat);
     float pw;
     if (POWMODE == 0) pw = r;
-    else if (POWMODE == 1) pw = __fsqrt_rn(r);
+    else if (POWMODE == 1) pw = WINDOW ? sqrt_in_range(r) : __fsqrt_rn(r);
     else pw = powf(r, p.hpow);
     const float den = __fadd_rn(pw, p.eps);
-    const float q = __fdiv_rn(mhat, den);
+    const float q = WINDOW && POWMODE != 2 ? div_in_range(mhat, den) : __fdiv_rn(mhat, den);
     if (WD) return __fsub_rn(x, __fmul_rn(p.lr, __fadd_rn(q, __fmul_rn(p.wd, x))));
     return __fsub_rn(x, __fmul_rn(p.lr, q));
 }
@@ -171,8 +174,8 @@ __device__ __forceinline__ void adahessian_update(float &x, float &m, float &v, 
 {
     moments(m, v, g, D, p);
     const float lo = fminf(fabsf(m), fabsf(v)), hi = fmaxf(fabsf(m), fabsf(v));
-    x = in_window(lo, hi) ? step_from_moments<POWMODE, WD, true>(x, m, v, p, w)
-                          : step_from_moments<POWMODE, WD, false>(x, m, v, p, w);
+    x = in_window(lo, hi) && p.narrow_ok ? step_from_moments<POWMODE, WD, true>(x, m, v, p, w)
+                                         : step_from_moments<POWMODE, WD, false>(x, m, v, p, w);
 }
 
 // Four consecutive elements at once: one window test for the eight divisions.
@@ -186,7 +189,7 @@ __device__ __forceinline__ void adahessian_update4(float4 &x, float4 &m, float4 
     moments(m.z, v.z, g.z, D.z, p);
     moments(m.w, v.w, g.w, D.w, p);
     const float lo = fminf(min_abs4(m), min_abs4(v)), hi = fmaxf(max_abs4(m), max_abs4(v));
-    if (in_window(lo, hi)) {
+    if (in_window(lo, hi) && p.narrow_ok) {
         x.x = step_from_moments<POWMODE, WD, true>(x.x, m.x, v.x, p, w);
         x.y = step_from_moments<POWMODE, WD, true>(x.y, m.y, v.y, p, w);
         x.z = step_from_moments<POWMODE, WD, true>(x.z, m.z, v.z, p, w);

@@ -61,6 +61,16 @@ def test_sample_z_bit_exact(B, torch, K, P):
     h.close()
 
 
+# ------------------------------------------------- premises of the exact arithmetic
+def test_branch_free_square_root_and_division_are_correctly_rounded(B, torch):
+    # the local step's square root and division inside the usual operand range are branch-free
+    # sequences built on hardware approximations; on this device: the square root equals the
+    # IEEE one for every input of its range, the refined reciprocal equals the IEEE reciprocal
+    # for every input of its range (the premise of Markstein's division), and the quotient
+    # equals the IEEE one on 2^33 seeded pairs, half of them aimed at rounding boundaries
+    assert B.ah_check_exact_arithmetic(1 << 33) == [0, 0, 0]
+
+
 # ---------------------------------------------------------------- local step
 @pytest.mark.parametrize("segs,P", [
     ([(0, 5000, 1)], 5000),                      # one unstructured tensor
