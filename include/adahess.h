@@ -226,8 +226,8 @@ int ah_sample_z_n(ah_ctx *h, uint64_t z_seed, uint32_t round, uint32_t sample, f
  * kernel: the tile sums climb a tree of arrival counters and whichever CTA completes the
  * last worker writes the K results to pinned host memory and, with AH_DIST_AND_RULE,
  * runs the weighting rule (u = log ||x_i - c||, Eqs. 10-11, h1 / h2 of Sec. V-B; same
- * bits as dw_weights_next).  A distance round therefore costs no launch of its own
- * (one more only when some workers sit the step out).
+ * bits as dw_weights_next).  A distance round therefore costs no launch of its own; a
+ * worker that sits the step out is measured by the same kernel (only its x is read).
  * A call that returns an error other than AH_ERR_CUDA leaves the handle unchanged.
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,

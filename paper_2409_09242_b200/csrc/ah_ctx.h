@@ -79,8 +79,6 @@ void commit_rule_in_round(ah_ctx *h, float alpha);
 int ring_to_host(ah_ctx *h);
 int ring_to_device(ah_ctx *h);
 int enqueue_weight_rule(ah_ctx *h, float alpha);   // ah_dynamic.cu
-cudaError_t launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows,
-                                 const DistTree &tree);   // ah_sgd.cu
 int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                   const uint16_t *order, const float *weights_dev, ExchangeParams &p);
 cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu

@@ -497,8 +497,6 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     const uint32_t calls = h->calls + 1;
     p.round = hy->round == AH_ROUND_AUTO ? calls : hy->round;
     p.nrows = 0;
-    uint16_t idle[AH_MAX_WORKERS];
-    uint32_t nidle = 0;
     uint32_t step[AH_MAX_WORKERS];                // step counts once this launch is enqueued
     for (int q = 0; q < h->K; ++q) {
         // a fused round walks the workers in their arrival order
@@ -511,10 +509,9 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         p.h2w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[i] : fx->alpha) : 0.f;
         p.h1w[i] = fx ? (fx->weights && !fx->lagged ? fx->weights[h->K + i] : fx->alpha) : 0.f;
         step[i] = h->step[i] + (on ? 1u : 0u);
-        // distances cover every worker; in a plain distance round the workers that sit
-        // the step out are measured by a streaming kernel of their own
-        if (on || meets || (dist && fx)) p.row[p.nrows++] = (uint16_t)i;
-        else if (dist) idle[nidle++] = (uint16_t)i;
+        // distances cover every worker: one that sits the step out travels through the
+        // pipeline as an item of its own that fetches only x and the master tile
+        if (on || meets || dist) p.row[p.nrows++] = (uint16_t)i;
         // bias corrections of Adam-type moments, 1 - beta^t with the worker's own t
         // (a worker that sat out steps has taken fewer); double, then one rounding
         const double t = (double)(step[i] ? step[i] : 1u);
@@ -547,10 +544,6 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
     if (fx && fx->dynamic) h->rule_fresh = false;     // the pending exchange has been made
     if (p.nitems) h->launches += 1;
-    if (nidle) {
-        AH_CUDA(h, launch_distance_rows(h, idle, nidle, p.tree));
-        h->launches += 1;
-    }
     if (dist) {
         const int rc = finish_distances(h);
         if (rc != AH_OK) return rc;

@@ -213,25 +213,6 @@ exchange_then_sgd_kernel(const __grid_constant__ SgdExchangeParams p)
 
 }  // namespace ah
 
-// Tile partials of ||x_i - c||^2 for workers that take no step this round (their x is
-// only read): the same streaming kernel with every listed row inactive.  Used by the
-// AdaHessian distance rounds so that stragglers do not travel through the local-step
-// pipeline one nearly empty item at a time.
-cudaError_t ah::launch_distance_rows(ah_ctx *h, const uint16_t *rows, uint32_t nrows,
-                                     const DistTree &tree)
-{
-    SgdParams p;
-    p.x = h->x; p.u = h->m; p.c = h->c; p.grad = nullptr;
-    p.tree = tree;
-    p.lds = h->lds; p.ld = 0;
-    p.P = h->P; p.ntiles = h->ntiles;
-    p.lr = 0.f; p.momentum = 0.f;
-    p.nrows = nrows;
-    for (int i = 0; i < h->K; ++i) p.active[i] = 0;
-    for (uint32_t r = 0; r < nrows; ++r) p.row[r] = rows[r];
-    return launch_sgd<false, true>(p, h->stream);
-}
-
 using namespace ah;
 
 extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const sgd_hyper *hy)

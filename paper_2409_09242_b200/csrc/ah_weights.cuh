@@ -18,31 +18,36 @@ struct WeightRule {
 // Pushes the sample u = log ||x_i - c|| into the worker's ring (newest first; the
 // first sample fills the whole ring), forms the raw score of Eqs. 10-11 and maps it
 // through h1 (worker-side coefficient) and h2 (master-side coefficient).
-__host__ __device__ inline void weight_rule_step(const WeightRule &r, double norm2, double *ring,
+__host__ __device__ inline void weight_rule_step(const WeightRule &rule, double norm2, double *ring,
                                                  bool ring_filled, float *to_master, float *to_worker)
 {
+    // the ring is read in one go (the loads do not wait for one another), moved on in
+    // registers and written back at the end
+    double past[AH_MAX_HIST + 1];
+    for (int j = 0; j <= rule.p_hist; ++j) past[j] = ring[j];
     const double u = u_from_norm2(norm2);
     if (ring_filled) {
-        for (int j = r.p_hist; j >= 1; --j) ring[j] = ring[j - 1];
+        for (int j = rule.p_hist; j >= 1; --j) past[j] = past[j - 1];
     } else {
-        for (int j = 1; j <= r.p_hist; ++j) ring[j] = u;
+        for (int j = 1; j <= rule.p_hist; ++j) past[j] = u;
     }
-    ring[0] = u;
+    past[0] = u;
     double score = 0.0;
-    for (int j = 0; j < r.p_hist; ++j)
-        score = AH_DADD(score, AH_DMUL(r.coef[j], AH_DSUB(ring[j], ring[j + 1])));
+    for (int j = 0; j < rule.p_hist; ++j)
+        score = AH_DADD(score, AH_DMUL(rule.coef[j], AH_DSUB(past[j], past[j + 1])));
+    for (int j = 0; j <= rule.p_hist; ++j) ring[j] = past[j];
     double w_worker, w_master;
-    if (score < r.kappa) {
+    if (score < rule.kappa) {
         w_worker = 1.0;
         w_master = 0.0;
     } else if (score <= 0.0) {
-        const double slope_worker = AH_DDIV(AH_DSUB(1.0, r.alpha), r.kappa);   // 1 -> alpha on [kappa, 0]
-        const double slope_master = AH_DDIV(-r.alpha, r.kappa);                // 0 -> alpha on [kappa, 0]
-        w_worker = AH_DADD(1.0, AH_DMUL(slope_worker, AH_DSUB(score, r.kappa)));
-        w_master = AH_DADD(AH_DMUL(slope_master, score), r.alpha);
+        const double slope_worker = AH_DDIV(AH_DSUB(1.0, rule.alpha), rule.kappa);   // 1 -> alpha on [kappa, 0]
+        const double slope_master = AH_DDIV(-rule.alpha, rule.kappa);                // 0 -> alpha on [kappa, 0]
+        w_worker = AH_DADD(1.0, AH_DMUL(slope_worker, AH_DSUB(score, rule.kappa)));
+        w_master = AH_DADD(AH_DMUL(slope_master, score), rule.alpha);
     } else {
-        w_worker = r.alpha;
-        w_master = r.alpha;
+        w_worker = rule.alpha;
+        w_master = rule.alpha;
     }
     *to_worker = (float)w_worker;
     *to_master = (float)w_master;
