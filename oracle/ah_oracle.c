@@ -20,8 +20,9 @@
  *
  * Parity pins (see tests): Philox known-answer vectors of Salmon et al. (SC'11);
  * Hutchinson identity on a diagonal quadratic (Sec. IV-B); reduction of the step to
- * Adam; closed forms of h1/h2 (Sec. V-B); EASGD reduction of Eqs. 12-13; a worked
- * two-worker example computed by hand in double precision.
+ * Adam, also for a worker that sits rounds out; closed forms of h1/h2 (Sec. V-B); the
+ * logarithm of u = log ||x_i - c|| against 300-bit arithmetic; EASGD reduction of
+ * Eqs. 12-13; a worked two-worker example computed by hand in double precision.
  *
  * Parity unpinned: the history depth p, the coefficients c_j and the threshold
  * (Sec. V-B gives no values) are run-time parameters; only their closed forms are

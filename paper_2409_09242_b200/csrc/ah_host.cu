@@ -705,7 +705,10 @@ int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device)
         AH_CUDA(h, cudaMemcpyAsync(&status, h->norm2_dev, sizeof(status), cudaMemcpyDeviceToHost,
                                    h->stream));
         AH_CUDA(h, cudaStreamSynchronize(h->stream));
-        if (status != 0u) return AH_ERR_INTERNAL;
+        if (status != 0u) {
+            h->tree_dirty = true;      // a kernel gave up half way: the next distance round starts clean
+            return AH_ERR_INTERNAL;
+        }
     }
     return state_copy(h, which, worker, dst, dst_on_device, true);
 }

@@ -1,6 +1,6 @@
-"""Pins for the oracle's own natural logarithm (double-double evaluation, used for
-u = log ||x_i - c||, Sec. V-B): against arbitrary-precision arithmetic, against the
-platform's libm, and at values that are known exactly."""
+"""Pins for the oracle's natural logarithm (the quad-precision library logarithm rounded
+once to double, used for u = log ||x_i - c||, Sec. V-B): against arbitrary-precision
+arithmetic, against the platform's libm, and at values that are known exactly."""
 import math
 
 import mpmath
