@@ -28,8 +28,6 @@ struct ah_ctx {
     ah::DistTree tree;             // the whole tree as the kernels see it (rule fields unset)
     size_t tree_count_bytes = 0;   // arrival counters (+ the finished-rows word) of the tree
     bool tree_dirty = false;       // a distance round failed half way: clear the counters first
-    ah::RuleConfig *rule_dev = nullptr;   // parameters of the weighting rule on the device
-    bool rule_dev_stale = true;    // ... no longer those of the host
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
     uint32_t *ring_flag_dev = nullptr;   // device copy of ring_filled

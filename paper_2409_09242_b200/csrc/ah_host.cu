@@ -37,7 +37,7 @@ int cuda_fail(ah_ctx *h, cudaError_t e)
     } while (0)
 
 struct Layout {
-    size_t x, m, v, c, partials, upper, count, norm2, sched, uhist, weights, rule, runs, tiles, total;
+    size_t x, m, v, c, partials, upper, count, norm2, sched, uhist, weights, runs, tiles, total;
     size_t count_bytes;
 };
 
@@ -85,7 +85,6 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.sched = take(4 * sizeof(uint32_t));                 // item counter, exit counter, ring flag
     L.uhist = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
     L.weights = take(2 * (size_t)K * sizeof(float));
-    L.rule = take(sizeof(RuleConfig));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
     L.total = off;
@@ -209,15 +208,10 @@ int ah::prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &
     if (run_rule) {
         const int rc = ring_to_device(h);
         if (rc != AH_OK) return rc;
-        if (h->rule_dev_stale) {
-            RuleConfig cfg;
-            memset(&cfg, 0, sizeof cfg);
-            for (int j = 0; j < h->p_hist; ++j) cfg.coef[j] = h->coef[j];
-            cfg.kappa = h->kappa;
-            cfg.p_hist = h->p_hist;
-            AH_CUDA(h, cudaMemcpyAsync(h->rule_dev, &cfg, sizeof cfg, cudaMemcpyHostToDevice, h->stream));
-            h->rule_dev_stale = false;
-        }
+        memset(&tree.rule, 0, sizeof tree.rule);
+        for (int j = 0; j < h->p_hist; ++j) tree.rule.coef[j] = h->coef[j];
+        tree.rule.kappa = h->kappa;
+        tree.rule.p_hist = h->p_hist;
     }
     h->tree_dirty = true;         // until finish_distances has seen every launch succeed
     return AH_OK;
@@ -354,8 +348,7 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->tree.norm2 = h->norm2_dev + 1;
     h->tree.norm2_host = h->norm2_host_dev;
     h->tree.status = reinterpret_cast<const uint32_t *>(h->norm2_dev);
-    h->rule_dev = (RuleConfig *)(base + L.rule);
-    h->tree.rule = h->rule_dev;
+    memset(&h->tree.rule, 0, sizeof h->tree.rule);
     h->tree.uhist = h->uhist_dev;
     h->tree.ring_flag = h->ring_flag_dev;
     h->tree.weights = h->weights_dev;
@@ -722,7 +715,6 @@ int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
     h->kappa = kappa;
     reset_history(h);
     h->ring_home = 0;
-    h->rule_dev_stale = true;
     return AH_OK;
 }
 

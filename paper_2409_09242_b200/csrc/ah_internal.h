@@ -89,8 +89,8 @@ struct WorkerConst {
     float bc1, bc2, rbc1, rbc2;
 };
 
-// Parameters of the weighting rule of Sec. V-B that change rarely (dw_config): kept in
-// the workspace for the kernels that run the rule at their end.
+// Parameters of the weighting rule of Sec. V-B (dw_config), as the kernels that run the
+// rule at their end receive them.
 struct RuleConfig {
     double coef[AH_MAX_HIST];  // c_0 .. c_{p-1}, c_0 on the newest difference
     double kappa;              // threshold of h1 / h2, negative
@@ -117,7 +117,7 @@ struct DistTree {
     double *norm2;                     // [K] roots
     double *norm2_host;                // pinned, mapped: [0] status word, [1 .. K] roots
     const uint32_t *status;            // device status word
-    const RuleConfig *rule;            // the rule at the end of the round: its parameters,
+    RuleConfig rule;                   // the rule at the end of the round: its parameters,
     double *uhist;                     //   the history ring [K][p + 1] on the device,
     uint32_t *ring_flag;               //   whether the ring has been filled,
     float *weights;                    //   and where the coefficients go: h2[K] then h1[K]

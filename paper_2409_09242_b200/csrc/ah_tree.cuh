@@ -31,9 +31,9 @@ static __device__ __noinline__ void finish_round(const DistTree &T, int lane)
     __syncwarp();
     WeightRule rule;
     if (T.run_rule) {
-        rule.p_hist = T.rule->p_hist;
-        for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < rule.p_hist ? T.rule->coef[j] : 0.0;
-        rule.kappa = T.rule->kappa;
+        rule.p_hist = T.rule.p_hist;
+        for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = T.rule.coef[j];
+        rule.kappa = T.rule.kappa;
         rule.alpha = T.rule_alpha;
     }
     for (uint32_t w = (uint32_t)lane; w < T.K; w += 32u) {
@@ -87,7 +87,7 @@ __device__ __forceinline__ uint32_t tree_count_tile(const DistTree &T, uint32_t 
 
 // Every lane with `climbing` set has just completed the level-1 node above its tile.  The
 // warp sums those nodes one after the other, all 32 lanes on one node at a time (two
-// children a lane, then the butterfly: the adjacent-pairs order; the loads of all the nodes
+// children a lane, then the butterfly: the adjacent-pairs order; the loads of eight nodes
 // are issued before the first sum is formed), delivers each to its parent, and repeats
 // with the lanes whose delivery completed the parent.  All 32 lanes must call; at the
 // top, whoever completes the last worker has the whole warp finish the round.
@@ -99,13 +99,13 @@ static __device__ __noinline__ void tree_climb(const DistTree &T, bool climbing,
     fence_gpu();                                       // counted children are visible from here on
     for (uint32_t todo = __ballot_sync(0xffffffffu, climbing); todo != 0u;
          todo = __ballot_sync(0xffffffffu, climbing)) {
-        // the nodes of this pass, four at a time: loads first, sums after
+        // the nodes of this pass, eight at a time: loads first, sums after
         double mine = 0.0;                             // lane e ends up with the sum of its own node
         for (uint32_t rest = todo; rest != 0u;) {
-            double pair[4];
-            int owner[4];
+            double pair[8];
+            int owner[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < 8; ++q) {
                 owner[q] = rest ? __ffs(rest) - 1 : -1;
                 if (rest) rest &= rest - 1u;
                 pair[q] = 0.0;
@@ -124,7 +124,7 @@ static __device__ __noinline__ void tree_climb(const DistTree &T, bool climbing,
                 }
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+            for (int q = 0; q < 8; ++q)
                 if (owner[q] >= 0) {
                     const double sum = warp_tree_sum(pair[q]);
                     if (lane == owner[q]) mine = sum;
