@@ -331,6 +331,23 @@ def test_async_rounds_resnet18_shape_reduced(B, torch):
     h.close()
 
 
+@pytest.mark.parametrize("K,width", [(40, 16), (256, 16)])
+def test_many_workers_with_the_rule_inside_the_distance_round(B, torch, K, width):
+    # more workers than lanes in a warp (the rule takes several workers per lane), the large
+    # per-worker launch tables, distances and rule inside the step kernel, the exchange riding on
+    # the next step: the shape the benchmark times for its largest worker counts
+    layout = W.resnet18_layout(width)
+    cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=12, tau=2,
+                    p_fail=0.2, max_stale=3, frozen=True, fused="next")
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, K, n_pool=2), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert log["exchanges"] == 6
+    h.close()
+
+
 # --------------------------------------- weights on the device, no host round trip
 @pytest.mark.parametrize("asyn,mode", [(False, "yes"), (True, "yes"), (False, "mixed"), (True, "mixed")])
 def test_dynamic_exchange_on_device_matches_oracle(B, torch, asyn, mode):
