@@ -275,8 +275,9 @@ def run_period(h, pool, t0, wl, events=None, stage=None, asynchronous=False, ex_
                                      order=h.dw_order_next(ORDER_SEED, t) if asynchronous else None,
                                      asynchronous=asynchronous, lagged=True, **HYPER)
         else:
-            # a distance round whose exchange will take its weights from the device also runs
-            # the weighting rule, in its last kernel
+            # a distance round whose exchange will take its weights from the device also asks
+            # for the weighting rule (it runs where the distances are assembled: at the head
+            # of the riding exchange, or in a small kernel of its own)
             rule = ex and (carry is not None or sync_free)
             h.ah_local_step(g, hv, Z_SEED, round_=t, active=mask if frozen else None,
                             want_dist=2 if rule else ex, rule_alpha=alpha,

@@ -92,12 +92,12 @@ typedef struct {
                              skips this step entirely (its x, m, v, step count stay)        */
     int want_dist;        /* AH_DIST: also compute n2_i = ||x_i - c||^2 after the step, for
                              all K workers, into the handle (read by dw_weights_next or by
-                             the device forms of the rule).  AH_DIST_AND_RULE: the kernel
-                             that completes the last distance also runs the weighting rule
-                             of Sec. V-B on the device with the moving rate rule_alpha; the
-                             next easgd_exchange_dynamic or easgd_exchange_then_step
-                             (dynamic != 0) with the same alpha uses its coefficients and
-                             launches no rule of its own.  AH_DIST_NONE: neither.          */
+                             the device forms of the rule).  AH_DIST_AND_RULE: the weighting
+                             rule of Sec. V-B is also owed on these distances, on the device,
+                             with the moving rate rule_alpha: it runs where the distances
+                             are assembled, and the next easgd_exchange_dynamic or
+                             easgd_exchange_then_step (dynamic != 0), which must name the
+                             same alpha, uses its coefficients.  AH_DIST_NONE: neither.    */
     int n_samples;        /* Hutchinson samples per step, 1 .. AH_MAX_SAMPLES; 0 means 1     */
     uint64_t hvp_sample_stride; /* elements from sample s to sample s + 1 inside hvp (a
                              multiple of 4, at least K * ld); ignored for one sample        */
@@ -222,12 +222,19 @@ int ah_sample_z_n(ah_ctx *h, uint64_t z_seed, uint32_t round, uint32_t sample, f
  * grad, hvp: device pointers, [K][ld] row-major, ld >= P, ld % 4 == 0, 16-byte
  * aligned, read only, must stay valid until the stream has run the step.
  * With hy->want_dist the squared distances ||x_i - c||^2 (binary32 difference,
- * squared and summed in double, pairwise order) are left in the handle, by the same
- * kernel: the tile sums climb a tree of arrival counters and whichever CTA completes the
- * last worker writes the K results to pinned host memory and, with AH_DIST_AND_RULE,
- * runs the weighting rule (u = log ||x_i - c||, Eqs. 10-11, h1 / h2 of Sec. V-B; same
- * bits as dw_weights_next).  A distance round therefore costs no launch of its own; a
- * worker that sits the step out is measured by the same kernel (only its x is read).
+ * squared and summed in double, pairwise order) are measured by the same kernel: it
+ * leaves one sum per worker and tile of 1024 parameters in the workspace (a worker that
+ * sits the step out is measured too: only its x is read).  The upper levels of the
+ * pairwise tree are formed by whoever needs the K distances next.  An exchange that
+ * rides on the next local step with the rule's coefficients (easgd_exchange_then_step,
+ * dynamic != 0; ah_local_step_exchange, lagged != 0) does it at the head of its own
+ * kernel, runs the weighting rule there (u = log ||x_i - c||, Eqs. 10-11, h1 / h2 of
+ * Sec. V-B; same bits as dw_weights_next) and leaves distances, coefficients and history
+ * where the other calls find them: between measuring the distances and using the
+ * coefficients lies no launch, no copy and no wait of the host.  Every other reader
+ * (dw_weights_next, easgd_exchange_dynamic, ah_state_get/set of the distances, the
+ * coefficients or the history, dw_config, the next distance round if a rule is still
+ * owed) first has a small kernel of its own assemble them.
  * A call that returns an error other than AH_ERR_CUDA leaves the handle unchanged.
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 int ah_local_step(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
@@ -445,6 +452,14 @@ int ah_check_exact_arithmetic(uint64_t division_pairs, uint64_t *mismatches, voi
  * Errors: INVALID_ARG, ALIGN, TOO_LARGE, CUDA. */
 int ah_distances_static(const float *x, uint64_t ldx, const float *c, int K, uint64_t P,
                         double *norm2, void *cuda_stream);
+
+/* How long the CTAs of a launch that assembles the distances of a round wait for one
+ * another, in polls of an arrival counter (roughly a microsecond each under load), before
+ * each of them forms the whole sum by itself (Sec. V-B: the K distances feed the rule).
+ * The distances do not depend on it: the sums follow one fixed tree whoever forms them.
+ * 0 makes every CTA work alone from the start.  Default 4096.  Host-side setting, takes
+ * effect with the next launch; returns AH_ERR_INVALID_ARG for a null handle. */
+int ah_set_wait_polls(ah_ctx *h, uint32_t polls);
 
 /* ---- diagnostics ------------------------------------------------------------- */
 const char *ah_status_string(int status);

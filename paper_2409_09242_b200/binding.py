@@ -37,7 +37,7 @@ EXPORTS = ["ah_workspace_bytes", "ah_init", "ah_destroy", "ah_state_set", "ah_st
            "ah_broadcast_center", "ah_sample_z", "ah_sample_z_n", "ah_local_step",
            "ah_local_step_exchange", "easgd_exchange_then_step", "dw_config",
            "dw_weights_next", "dw_weights_from_norm2", "dw_mask_next", "easgd_exchange",
-           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "easgd_exchange_then_sgd_step", "dw_partition", "ah_distances_static", "ah_check_exact_arithmetic", "ah_status_string",
+           "dw_order_next", "easgd_exchange_async", "easgd_exchange_dynamic", "sgd_local_step", "easgd_exchange_then_sgd_step", "dw_partition", "ah_distances_static", "ah_check_exact_arithmetic", "ah_set_wait_polls", "ah_status_string",
            "ah_last_cuda_error", "ah_launch_count"]
 
 
@@ -97,6 +97,7 @@ _lib.easgd_exchange_dynamic.argtypes = [_vp, C.POINTER(C.c_uint8), C.c_float, C.
                                         C.c_int]
 _lib.ah_distances_static.argtypes = [_vp, C.c_uint64, _vp, C.c_int, C.c_uint64, _vp, _vp]
 _lib.ah_check_exact_arithmetic.argtypes = [C.c_uint64, C.POINTER(C.c_uint64), _vp]
+_lib.ah_set_wait_polls.argtypes = [_vp, C.c_uint32]
 _lib.ah_status_string.argtypes = [C.c_int]
 _lib.ah_status_string.restype = C.c_char_p
 _lib.ah_last_cuda_error.argtypes = [_vp]
@@ -519,6 +520,9 @@ class Handle:
             o = order.ctypes.data_as(C.POINTER(C.c_uint16))
         self._check(_lib.easgd_exchange_dynamic(self._h, m, alpha, o, 1 if asynchronous else 0),
                     "easgd_exchange_dynamic")
+
+    def ah_set_wait_polls(self, polls):
+        self._check(_lib.ah_set_wait_polls(self._h, int(polls)), "ah_set_wait_polls")
 
     def ah_launch_count(self):
         return int(_lib.ah_launch_count(self._h))

@@ -24,14 +24,16 @@ struct ah_ctx {
 
     // device views into the workspace
     float *x = nullptr, *m = nullptr, *v = nullptr, *c = nullptr;
-    double *partials = nullptr;    // level 0 of the distance tree: [K][ntiles_pad]
-    ah::DistTree tree;             // the whole tree as the kernels see it (rule fields unset)
-    size_t tree_count_bytes = 0;   // arrival counters (+ the finished-rows word) of the tree
-    bool tree_dirty = false;       // a distance round failed half way: clear the counters first
+    double *sums[2] = {nullptr, nullptr};   // level 0 of the distance tree, two copies: [K][ntiles_pad]
+    int sums_cur = 0;              // the copy that holds the latest distance round's tile sums
+    ah::DistTree tree;             // the tree's shape and fixed addresses (per-launch fields unset)
+    uint32_t arrive_total = 0;     // what the tree's arrival counters stand at
+    bool tree_dirty = false;       // a kernel gave up half way: clear the arrival counters first
+    uint32_t wait_polls = 4096;    // how long the CTAs of an assembling launch wait for one another
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
-    uint32_t *ring_flag_dev = nullptr;   // device copy of ring_filled
-    double *uhist_dev = nullptr;   // device copy of the history ring, [K][p_hist + 1]
+    double *ring_dev[2] = {nullptr, nullptr};   // device copies of the history ring, [K][p_hist + 1]:
+    int ring_cur = 0;              //   a rule on the device reads ring_dev[ring_cur] and writes the other
     float *weights_dev = nullptr;  // [2K] coefficients of the last dynamic exchange
     ah::Run *runs = nullptr;
     ah::TileInfo *tiles = nullptr;
@@ -39,16 +41,21 @@ struct ah_ctx {
 
     // host state
     double *norm2_host = nullptr;  // pinned, mapped copy of norm2_dev (status word + K doubles):
-                                   // written by the kernel that completes the last distance
+                                   // written by the launch that assembles the distances
     double *norm2_host_dev = nullptr;   // the same memory as the device addresses it
     cudaEvent_t norm2_ready = nullptr;
+    bool sums_raw = false;         // the latest distance round's tile sums wait in sums[sums_cur]:
+                                   // nobody has assembled them yet
+    bool raw_rule = false;         // ... and whoever assembles them also runs the weighting rule,
+    float raw_alpha = 0.f;         //     with this moving rate
     bool norm2_pending = false;    // distances of a want_dist step not yet used by a weight rule
     bool norm2_unread = false;     // ... and not yet copied into norm2_last
     int ring_home = 0;             // 0: the host copy of the ring is current, 1: the device copy
     bool lagged_ready = false;     // weights_dev holds the rule's output of an earlier fused round
-    bool rule_fresh = false;       // weights_dev holds the rule's output for the distances of the
-                                   // last want_dist step (AH_DIST_AND_RULE), not yet used
-    float rule_fresh_alpha = 0.f;  // ... computed with this moving rate
+    bool rule_fresh = false;       // the rule's output for the distances of the last want_dist
+                                   // step (AH_DIST_AND_RULE) is owed to the next exchange (it is in
+                                   // weights_dev once those distances have been assembled)
+    float rule_fresh_alpha = 0.f;  // ... with this moving rate
     double norm2_last[AH_MAX_WORKERS];
     uint32_t step[AH_MAX_WORKERS];
     uint32_t down_until[AH_MAX_WORKERS];
@@ -71,13 +78,17 @@ inline int ah_cuda_fail(ah_ctx *h, cudaError_t e)
 }
 
 namespace ah {
-int finish_distances(ah_ctx *h);   // ah_host.cu
-int prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &tree);
-void commit_rule_in_round(ah_ctx *h, float alpha);
+// ah_host.cu: the life of a distance round's tile sums
+int begin_distance_store(ah_ctx *h, DistTree &tree);       // a launch is about to store a round's sums
+void commit_distance_store(ah_ctx *h, bool rule, float alpha, bool owed_to_exchange);
+int begin_assembly(ah_ctx *h, bool run_rule, float alpha, uint32_t sync_ctas, DistTree &tree);
+int commit_assembly(ah_ctx *h, const DistTree &tree);
+int settle_distances(ah_ctx *h);   // assembles waiting sums with a kernel of its own, if any
 int ring_to_host(ah_ctx *h);
 int ring_to_device(ah_ctx *h);
 int enqueue_weight_rule(ah_ctx *h, float alpha);   // ah_dynamic.cu
 int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                   const uint16_t *order, const float *weights_dev, ExchangeParams &p);
 cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu
+cudaError_t launch_assemble(const DistTree &T, cudaStream_t s);                  // ah_kernels.cu
 }

@@ -11,42 +11,41 @@ namespace ah {
 // entry points run), on the device copy of the history ring.
 __global__ void __launch_bounds__(AH_MAX_WORKERS)
 dynamic_weights_kernel(const __grid_constant__ WeightRule rule, const double *norm2, double *uhist,
-                       uint32_t *ring_flag, float *weights, int nworkers)
+                       bool filled, float *weights, int nworkers)
 {
     const int i = threadIdx.x;
-    const bool filled = *ring_flag != 0u;
-    __syncthreads();                               // everybody has read the flag
-    if (i < nworkers)
-        weight_rule_step(rule, norm2[i], uhist + (size_t)i * (rule.p_hist + 1), filled, &weights[i],
-                         &weights[nworkers + i]);
-    if (i == 0) *ring_flag = 1u;
+    if (i < nworkers) {
+        double *ring = uhist + (size_t)i * (rule.p_hist + 1);
+        weight_rule_step(rule, norm2[i], ring, ring, filled, &weights[i], &weights[nworkers + i]);
+    }
 }
 
 }  // namespace ah
 
 using namespace ah;
 
-// The weighting rule on the device, fed by the distances the last want_dist step left
-// there; its coefficients stay in weights_dev.
+// The weighting rule on the device, fed by assembled distances that wait in norm2_dev
+// (restored from a snapshot, or assembled for another reader before the exchange asked
+// for coefficients); its coefficients stay in weights_dev.
 int ah::enqueue_weight_rule(ah_ctx *h, float alpha)
 {
     const int rc = ring_to_device(h);
     if (rc != AH_OK) return rc;
+    const bool filled = h->ring_home == 1 || h->ring_filled != 0;
     WeightRule rule;
     rule.p_hist = h->p_hist;
     for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < h->p_hist ? h->coef[j] : 0.0;
     rule.kappa = h->kappa;
     rule.alpha = (double)alpha;
-    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1, h->uhist_dev,
-                                                                 h->ring_flag_dev, h->weights_dev, h->K);
+    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1,
+                                                                 h->ring_dev[h->ring_cur], filled,
+                                                                 h->weights_dev, h->K);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return ah_cuda_fail(h, e);
     h->launches += 1;
     h->ring_home = 1;                              // the device copy of the ring leads
     h->norm2_pending = false;                      // these distances have fed the rule
     h->lagged_ready = true;                        // weights_dev now holds coefficients
-    h->rule_fresh = true;                          // ... of the exchange that is still to come
-    h->rule_fresh_alpha = alpha;
     return AH_OK;
 }
 
@@ -55,8 +54,9 @@ extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, flo
 {
     if (!h) return AH_ERR_INVALID_ARG;
     if (!h->has_device) return AH_ERR_STATE;
-    // the rule has either run already at the end of the distance round (its output is
-    // waiting in weights_dev), or runs now on the pending distances
+    // the rule is either owed on the last distance round (AH_DIST_AND_RULE) or runs now on
+    // the pending distances; either way it goes with the assembly of that round's tile
+    // sums if they still wait, and its output ends up in weights_dev
     if (h->rule_fresh) {
         if (alpha != h->rule_fresh_alpha) return AH_ERR_INVALID_ARG;
     } else if (!h->norm2_pending) {
@@ -66,7 +66,12 @@ extern "C" int easgd_exchange_dynamic(ah_ctx *h, const uint8_t *worker_mask, flo
     int rc = fill_exchange(h, worker_mask, nullptr, alpha, asynchronous ? order : nullptr,
                            h->weights_dev, p);
     if (rc != AH_OK) return rc;
-    if (!h->rule_fresh && (rc = enqueue_weight_rule(h, alpha)) != AH_OK) return rc;
+    if (h->sums_raw && !h->raw_rule) {
+        h->raw_rule = true;
+        h->raw_alpha = alpha;
+    }
+    if ((rc = settle_distances(h)) != AH_OK) return rc;
+    if (!h->rule_fresh && h->norm2_pending && (rc = enqueue_weight_rule(h, alpha)) != AH_OK) return rc;
     if (p.nact == 0) {                             // the history advances even if nobody arrives
         h->rule_fresh = false;
         return AH_OK;

@@ -37,14 +37,14 @@ int cuda_fail(ah_ctx *h, cudaError_t e)
     } while (0)
 
 struct Layout {
-    size_t x, m, v, c, partials, upper, count, norm2, sched, uhist, weights, runs, tiles, total;
-    size_t count_bytes;
+    size_t x, m, v, c, sums[2], upper, arrive, norm2, sched, ring[2], weights, runs, tiles, total;
 };
 
 // Shape of the distance tree over ntp = 2^a tile slots of which ntiles exist: nodes per
-// worker at every level, how many of them are live, and where each level starts.  Returns
-// the nodes per worker above level 0.
-uint32_t tree_shape(uint32_t ntiles, uint32_t ntp, DistTree &T)
+// worker at every level, how many of them are live, where each level starts, and which
+// levels are large enough (over all K workers) to be shared between CTAs.  Returns the
+// nodes per worker above level 0.
+uint32_t tree_shape(uint32_t ntiles, uint32_t ntp, uint32_t K, DistTree &T)
 {
     T.n[0] = ntp;
     T.live[0] = ntiles;
@@ -59,6 +59,10 @@ uint32_t tree_shape(uint32_t ntiles, uint32_t ntp, DistTree &T)
     } while (T.n[L] > 1u);
     T.levels = L;
     for (uint32_t q = L + 1; q <= (uint32_t)kTreeMaxLevels; ++q) T.n[q] = T.live[q] = T.off[q] = 0u;
+    T.K = K;
+    T.shared_levels = 0;
+    for (uint32_t q = 1; q <= L; ++q)
+        if ((uint64_t)K * T.live[q - 1] > kTreeOwnLevelInputs) T.shared_levels = q;
     return above;
 }
 
@@ -75,15 +79,16 @@ Layout workspace_layout(int K, uint64_t P, int nruns_max)
     L.m = take((size_t)K * lds * sizeof(float));
     L.v = take((size_t)K * lds * sizeof(float));
     L.c = take((size_t)lds * sizeof(float));
-    L.partials = take((size_t)K * ntp * sizeof(double));
+    L.sums[0] = take((size_t)K * ntp * sizeof(double));
+    L.sums[1] = take((size_t)K * ntp * sizeof(double));
     DistTree shape;
-    const uint32_t above = tree_shape(ntiles, ntp, shape);
+    const uint32_t above = tree_shape(ntiles, ntp, (uint32_t)K, shape);
     L.upper = take((size_t)K * above * sizeof(double));
-    L.count_bytes = ((size_t)K * above + 1) * sizeof(uint32_t);     // + the finished-rows word
-    L.count = take(L.count_bytes);
+    L.arrive = take((kTreeMaxLevels + 1) * sizeof(uint32_t));
     L.norm2 = take((size_t)(AH_MAX_WORKERS + 1) * sizeof(double));
-    L.sched = take(4 * sizeof(uint32_t));                 // item counter, exit counter, ring flag
-    L.uhist = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
+    L.sched = take(4 * sizeof(uint32_t));                 // item counter, exit counter
+    L.ring[0] = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
+    L.ring[1] = take((size_t)K * (AH_MAX_HIST + 1) * sizeof(double));
     L.weights = take(2 * (size_t)K * sizeof(float));
     L.runs = take((size_t)nruns_max * sizeof(Run));
     L.tiles = take((size_t)ntiles * sizeof(TileInfo));
@@ -161,18 +166,21 @@ void reset_history(ah_ctx *h)
 
 }  // namespace
 
-// The history ring of the weighting rule has a host copy and a device copy; ring_home
-// says which one is current.  These bring the other side up to date.
+// The history ring of the weighting rule has a host copy and device copies; ring_home
+// says which side is current.  These bring the other side up to date.  A rule that is
+// still owed on waiting tile sums runs first: it belongs in front of whatever looks at
+// the ring next.
 int ah::ring_to_host(ah_ctx *h)
 {
-    if (!h->has_device || h->ring_home == 0) return AH_OK;
+    if (!h->has_device) return AH_OK;
+    const int rc = settle_distances(h);
+    if (rc != AH_OK) return rc;
+    if (h->ring_home == 0) return AH_OK;
     AH_CUDA(h, cudaStreamSynchronize(h->stream));
     const size_t depth = (size_t)h->p_hist + 1;
-    AH_CUDA(h, cudaMemcpy(h->uhist.data(), h->uhist_dev, (size_t)h->K * depth * sizeof(double),
+    AH_CUDA(h, cudaMemcpy(h->uhist.data(), h->ring_dev[h->ring_cur], (size_t)h->K * depth * sizeof(double),
                           cudaMemcpyDeviceToHost));
-    uint32_t filled = 0;
-    AH_CUDA(h, cudaMemcpy(&filled, h->ring_flag_dev, sizeof(filled), cudaMemcpyDeviceToHost));
-    h->ring_filled = (int)filled;
+    h->ring_filled = 1;           // a rule has run on the device
     h->ring_home = 0;
     return AH_OK;
 }
@@ -184,25 +192,55 @@ int ah::ring_to_device(ah_ctx *h)
 {
     if (h->ring_home == 1) return AH_OK;
     const size_t depth = (size_t)h->p_hist + 1;
-    const uint32_t filled = (uint32_t)h->ring_filled;
-    // pageable sources: the calls return once the data has been staged
-    AH_CUDA(h, cudaMemcpyAsync(h->uhist_dev, h->uhist.data(), (size_t)h->K * depth * sizeof(double),
-                               cudaMemcpyHostToDevice, h->stream));
-    AH_CUDA(h, cudaMemcpyAsync(h->ring_flag_dev, &filled, sizeof(filled), cudaMemcpyHostToDevice,
-                               h->stream));
+    // pageable source: the call returns once the data has been staged
+    AH_CUDA(h, cudaMemcpyAsync(h->ring_dev[h->ring_cur], h->uhist.data(),
+                               (size_t)h->K * depth * sizeof(double), cudaMemcpyHostToDevice, h->stream));
     return AH_OK;
 }
 
-// What a launch that measures distances needs to know about the tree.  With run_rule the
-// kernel that completes the last distance also runs the weighting rule (moving rate
-// alpha) on the device copy of the history, which is brought up to date first.
-int ah::prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &tree)
+// A launch is about to store a distance round's tile sums: they go to the copy of level 0
+// that holds nothing anybody still needs.
+int ah::begin_distance_store(ah_ctx *h, DistTree &tree)
 {
-    if (h->tree_dirty) {          // an earlier distance round stopped half way
-        AH_CUDA(h, cudaMemsetAsync(h->tree.count, 0, h->tree_count_bytes, h->stream));
+    // sums of an earlier round that nobody has assembled: if a rule is owed on them it
+    // runs now (the history advances once per such round); otherwise they are superseded
+    if (h->sums_raw && h->raw_rule && !tree.assemble) {
+        const int rc = settle_distances(h);
+        if (rc != AH_OK) return rc;
+    }
+    tree.sums_out = h->sums[h->sums_cur ^ 1];
+    return AH_OK;
+}
+
+// ... and has been enqueued.  `rule`: whoever assembles these sums also runs the weighting
+// rule with moving rate alpha; `owed_to_exchange`: its output belongs to the next exchange
+// (AH_DIST_AND_RULE).
+void ah::commit_distance_store(ah_ctx *h, bool rule, float alpha, bool owed_to_exchange)
+{
+    h->sums_cur ^= 1;
+    h->sums_raw = true;
+    h->raw_rule = rule;
+    h->raw_alpha = alpha;
+    h->norm2_pending = true;
+    h->norm2_unread = true;
+    h->rule_fresh = owed_to_exchange;
+    if (owed_to_exchange) h->rule_fresh_alpha = alpha;
+}
+
+// A launch is about to assemble the waiting tile sums at its head (its first sync_ctas
+// CTAs share the large levels), and to run the weighting rule on the result if asked.
+int ah::begin_assembly(ah_ctx *h, bool run_rule, float alpha, uint32_t sync_ctas, DistTree &tree)
+{
+    if (h->tree_dirty) {          // an earlier kernel stopped half way
+        AH_CUDA(h, cudaMemsetAsync(h->tree.arrive, 0, (kTreeMaxLevels + 1) * sizeof(uint32_t), h->stream));
+        h->arrive_total = 0;
         h->tree_dirty = false;
     }
-    tree = h->tree;
+    tree.assemble = 1u;
+    tree.sums_in = h->sums[h->sums_cur];
+    tree.sync_ctas = sync_ctas;
+    tree.arrive_target = h->arrive_total + sync_ctas;
+    tree.wait_polls = h->wait_polls;
     tree.run_rule = run_rule ? 1u : 0u;
     tree.rule_alpha = (double)alpha;
     if (run_rule) {
@@ -212,31 +250,46 @@ int ah::prepare_distance_round(ah_ctx *h, bool run_rule, float alpha, DistTree &
         for (int j = 0; j < h->p_hist; ++j) tree.rule.coef[j] = h->coef[j];
         tree.rule.kappa = h->kappa;
         tree.rule.p_hist = h->p_hist;
+        tree.ring_in = h->ring_dev[h->ring_cur];
+        tree.ring_out = h->ring_dev[h->ring_cur ^ 1];
+        tree.ring_filled = h->ring_home == 1 ? 1u : (uint32_t)(h->ring_filled != 0);
     }
-    h->tree_dirty = true;         // until finish_distances has seen every launch succeed
     return AH_OK;
 }
 
-// Bookkeeping after a round whose last kernel also ran the weighting rule.
-void ah::commit_rule_in_round(ah_ctx *h, float alpha)
+// ... and has been enqueued: the K doubles (and the status word in front of them) will be
+// in pinned host memory once it has run, so an event behind it is all the host needs to
+// wait for; the rule's bookkeeping follows.
+int ah::commit_assembly(ah_ctx *h, const DistTree &tree)
 {
-    h->ring_home = 1;             // the device copy of the ring leads
-    h->norm2_pending = false;     // these distances have fed the rule
-    h->lagged_ready = true;       // weights_dev holds coefficients
-    h->rule_fresh_alpha = alpha;
-}
-
-// After every kernel of a distance round has been enqueued: the kernel that completes
-// the last distance leaves the K doubles (and the status word in front of them) in pinned
-// host memory, so an event behind it is all the host needs to wait for.
-int ah::finish_distances(ah_ctx *h)
-{
+    h->arrive_total = tree.arrive_target;
+    h->sums_raw = false;
+    if (tree.run_rule) {
+        h->ring_cur ^= 1;
+        h->ring_home = 1;         // the device copy of the ring leads
+        h->norm2_pending = false; // these distances have fed the rule
+        h->lagged_ready = true;   // weights_dev holds coefficients
+    }
     AH_CUDA(h, cudaEventRecord(h->norm2_ready, h->stream));
-    h->tree_dirty = false;
-    h->norm2_pending = true;
-    h->norm2_unread = true;
-    h->rule_fresh = false;
     return AH_OK;
+}
+
+// Readers other than a fused exchange: the waiting sums are assembled by a small kernel
+// of its own (and the rule that is owed on them runs there).
+int ah::settle_distances(ah_ctx *h)
+{
+    if (!h->has_device || !h->sums_raw) return AH_OK;
+    DistTree tree = h->tree;
+    // one warp a node of the first level, four warps a CTA, at most one CTA per SM
+    const uint64_t nodes = (uint64_t)h->K * tree.live[1];
+    uint32_t ctas = (uint32_t)((nodes + 3) / 4);
+    if (ctas > (uint32_t)h->sm_count) ctas = (uint32_t)h->sm_count;
+    if (ctas < 1u) ctas = 1u;
+    const int rc = begin_assembly(h, h->raw_rule, h->raw_alpha, ctas, tree);
+    if (rc != AH_OK) return rc;
+    AH_CUDA(h, launch_assemble(tree, h->stream));
+    h->launches += 1;
+    return commit_assembly(h, tree);
 }
 
 extern "C" {
@@ -316,11 +369,12 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
     h->m = (float *)(base + L.m);
     h->v = (float *)(base + L.v);
     h->c = (float *)(base + L.c);
-    h->partials = (double *)(base + L.partials);
+    h->sums[0] = (double *)(base + L.sums[0]);
+    h->sums[1] = (double *)(base + L.sums[1]);
     h->norm2_dev = (double *)(base + L.norm2);
     h->sched = (uint32_t *)(base + L.sched);
-    h->ring_flag_dev = h->sched + 2;
-    h->uhist_dev = (double *)(base + L.uhist);
+    h->ring_dev[0] = (double *)(base + L.ring[0]);
+    h->ring_dev[1] = (double *)(base + L.ring[1]);
     h->weights_dev = (float *)(base + L.weights);
     h->runs = (Run *)(base + L.runs);
     h->tiles = (TileInfo *)(base + L.tiles);
@@ -338,23 +392,15 @@ int ah_init(ah_ctx **out, int K, uint64_t P, const ah_segment *segs, int nseg, c
         return fail(AH_ERR_ALLOC);
     }
     memset(h->norm2_host, 0, (AH_MAX_WORKERS + 1) * sizeof(double));
-    // the distance tree as the kernels see it
-    tree_shape(h->ntiles, h->ntiles_pad, h->tree);
-    h->tree.level0 = h->partials;
+    // the distance tree as the kernels see it: shape and fixed addresses
+    memset(&h->tree, 0, sizeof h->tree);
+    tree_shape(h->ntiles, h->ntiles_pad, (uint32_t)K, h->tree);
     h->tree.upper = (double *)(base + L.upper);
-    h->tree.count = (uint32_t *)(base + L.count);
-    h->tree.rows_done = h->tree.count + (L.count_bytes / sizeof(uint32_t) - 1);
-    h->tree_count_bytes = L.count_bytes;
+    h->tree.arrive = (uint32_t *)(base + L.arrive);
     h->tree.norm2 = h->norm2_dev + 1;
     h->tree.norm2_host = h->norm2_host_dev;
     h->tree.status = reinterpret_cast<const uint32_t *>(h->norm2_dev);
-    memset(&h->tree.rule, 0, sizeof h->tree.rule);
-    h->tree.uhist = h->uhist_dev;
-    h->tree.ring_flag = h->ring_flag_dev;
     h->tree.weights = h->weights_dev;
-    h->tree.rule_alpha = 0.0;
-    h->tree.run_rule = 0u;
-    h->tree.K = (uint32_t)K;
     // state (and its row padding) starts at zero; descriptors go up once
     if ((e = cudaMemsetAsync(h->workspace, 0, L.runs, h->stream)) != cudaSuccess ||
         (e = cudaMemcpyAsync(h->runs, runs.data(), runs.size() * sizeof(Run), cudaMemcpyHostToDevice,
@@ -451,8 +497,8 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         }
     }
     const bool dist = hy->want_dist != AH_DIST_NONE;
-    // the weighting rule at the end of this round's last kernel: asked for by the caller,
-    // or (lagged one-pass rounds) to serve the next exchange round
+    // the weighting rule owed on this round's distances: asked for by the caller, or
+    // (lagged one-pass rounds) to serve the next exchange round
     const bool rule_here = hy->want_dist == AH_DIST_AND_RULE || (fx && fx->lagged && dist);
     const float rule_alpha = hy->want_dist == AH_DIST_AND_RULE ? hy->rule_alpha : (fx ? fx->alpha : 0.f);
     if (hy->want_dist == AH_DIST_AND_RULE && fx && !fx->lagged) return AH_ERR_INVALID_ARG;
@@ -486,6 +532,8 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     p.any_exchange = 0u;
     p.nworkers = (uint32_t)h->K;
     p.c_out = h->c;
+    // coefficients from the device: read from weights_dev unless this launch forms them
+    // itself at its head (see below)
     p.wdev = fx && ((fx->lagged && h->lagged_ready) || fx->dynamic) ? h->weights_dev : nullptr;
     const uint32_t calls = h->calls + 1;
     p.round = hy->round == AH_ROUND_AUTO ? calls : hy->round;
@@ -522,29 +570,52 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
         if (!(p.w[i].bc1 >= 0x1p-24f && p.w[i].bc2 >= 0x1p-24f)) p.narrow_ok = 0u;
 
     // ---- enqueue; the handle's bookkeeping follows each launch that went in
-    if (fx && fx->dynamic && !h->rule_fresh) {
-        const int rc = enqueue_weight_rule(h, fx->alpha);
+    // Tile sums of the last distance round may still wait to be assembled.  A fused exchange
+    // that takes its coefficients from the device does that at the head of its own kernel
+    // (and runs the rule there); every other reader gets a small kernel of its own.
+    bool assemble_here = false, rule_at_head = false;
+    float head_alpha = 0.f;
+    if (fx && h->sums_raw && p.nitems > 0) {
+        if (fx->dynamic) {
+            assemble_here = rule_at_head = true;
+            head_alpha = h->rule_fresh ? h->rule_fresh_alpha : fx->alpha;
+        } else if (fx->lagged && h->raw_rule) {
+            assemble_here = rule_at_head = true;
+            head_alpha = h->raw_alpha;
+        }
+    }
+    if (fx && fx->dynamic && !assemble_here) {
+        if (h->sums_raw && !h->raw_rule) {        // the rule goes with the assembly
+            h->raw_rule = true;
+            h->raw_alpha = fx->alpha;
+        }
+        int rc = settle_distances(h);
+        if (rc != AH_OK) return rc;
+        if (!h->rule_fresh && h->norm2_pending && (rc = enqueue_weight_rule(h, fx->alpha)) != AH_OK)
+            return rc;
+    }
+    p.tree = h->tree;
+    if (assemble_here) {
+        // its first CTAs share the large levels: the grid has at least this many
+        const uint32_t sync_ctas = p.nitems < (uint32_t)h->sm_count ? p.nitems : (uint32_t)h->sm_count;
+        const int rc = begin_assembly(h, rule_at_head, head_alpha, sync_ctas, p.tree);
         if (rc != AH_OK) return rc;
     }
     if (dist) {
-        const int rc = prepare_distance_round(h, rule_here, rule_alpha, p.tree);
+        const int rc = begin_distance_store(h, p.tree);
         if (rc != AH_OK) return rc;
-    } else {
-        memset(&p.tree, 0, sizeof p.tree);
     }
     AH_CUDA(h, launch_local_step(p, dist, h->sm_count, h->stream));
     h->calls = calls;
     memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
-    if (fx && fx->dynamic) h->rule_fresh = false;     // the pending exchange has been made
     if (p.nitems) h->launches += 1;
-    if (dist) {
-        const int rc = finish_distances(h);
+    if (assemble_here) {
+        const int rc = commit_assembly(h, p.tree);
         if (rc != AH_OK) return rc;
-        if (rule_here) {
-            commit_rule_in_round(h, rule_alpha);
-            h->rule_fresh = hy->want_dist == AH_DIST_AND_RULE;
-        }
     }
+    if (fx && fx->dynamic) h->rule_fresh = false;     // the pending exchange has been made
+    if (dist && p.nitems)
+        commit_distance_store(h, rule_here, rule_alpha, hy->want_dist == AH_DIST_AND_RULE);
     return AH_OK;
 }
 
@@ -609,6 +680,12 @@ static int state_copy(ah_ctx *h, int which, int worker, void *user, int on_devic
         return AH_OK;
     }
     if (on_device) return AH_ERR_INVALID_ARG;
+    if (which == AH_WEIGHTS || which == AH_NORM2 || which == AH_UHIST || which == AH_ROUND) {
+        // tile sums that still wait are assembled first (and the rule owed on them runs):
+        // these selectors show, or replace, what that leaves behind
+        const int rc = settle_distances(h);
+        if (rc != AH_OK) return rc;
+    }
     if (which == AH_WEIGHTS) {                 // coefficients of the last rule run on the device
         if (!h->has_device) return AH_ERR_STATE;
         if (to_user) {
@@ -710,6 +787,8 @@ int ah_state_get(ah_ctx *h, int which, int worker, void *dst, int dst_on_device)
 int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
 {
     if (!h || !c || p_hist < 1 || p_hist > AH_MAX_HIST || !(kappa < 0.0)) return AH_ERR_INVALID_ARG;
+    const int rc = settle_distances(h);        // a rule that is still owed runs with the old setting
+    if (rc != AH_OK) return rc;
     h->p_hist = p_hist;
     for (int j = 0; j < p_hist; ++j) h->coef[j] = c[j];
     h->kappa = kappa;
@@ -721,7 +800,10 @@ int dw_config(ah_ctx *h, int p_hist, const double *c, double kappa)
 int dw_weights_next(ah_ctx *h, float alpha, float *weights)
 {
     if (!h || !weights) return AH_ERR_INVALID_ARG;
-    if (!h->has_device || !h->norm2_pending) return AH_ERR_STATE;
+    if (!h->has_device) return AH_ERR_STATE;
+    const int rc = settle_distances(h);
+    if (rc != AH_OK) return rc;
+    if (!h->norm2_pending) return AH_ERR_STATE;
     AH_CUDA(h, cudaEventSynchronize(h->norm2_ready));
     h->norm2_pending = false;
     h->norm2_unread = false;
@@ -742,9 +824,11 @@ int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *we
     rule.kappa = h->kappa;
     rule.alpha = (double)alpha;
     const int depth = h->p_hist + 1;
-    for (int i = 0; i < h->K; ++i)
-        weight_rule_step(rule, h->norm2_last[i], &h->uhist[(size_t)i * depth], h->ring_filled != 0,
-                         &weights[i], &weights[h->K + i]);
+    for (int i = 0; i < h->K; ++i) {
+        double *ring = &h->uhist[(size_t)i * depth];
+        weight_rule_step(rule, h->norm2_last[i], ring, ring, h->ring_filled != 0, &weights[i],
+                         &weights[h->K + i]);
+    }
     h->ring_filled = 1;
     return AH_OK;
 }
@@ -807,6 +891,13 @@ const char *ah_status_string(int status)
     case AH_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity";
     default: return "unknown status";
     }
+}
+
+int ah_set_wait_polls(ah_ctx *h, uint32_t polls)
+{
+    if (!h) return AH_ERR_INVALID_ARG;
+    h->wait_polls = polls;
+    return AH_OK;
 }
 
 int ah_last_cuda_error(const ah_ctx *h) { return h ? h->last_cuda : 0; }

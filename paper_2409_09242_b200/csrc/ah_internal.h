@@ -90,7 +90,7 @@ struct WorkerConst {
 };
 
 // Parameters of the weighting rule of Sec. V-B (dw_config), as the kernels that run the
-// rule at their end receive them.
+// rule after assembling the distances receive them.
 struct RuleConfig {
     double coef[AH_MAX_HIST];  // c_0 .. c_{p-1}, c_0 on the newest difference
     double kappa;              // threshold of h1 / h2, negative
@@ -98,31 +98,45 @@ struct RuleConfig {
     int reserved;
 };
 
-// Where the squared distances ||x_i - c||^2 of a round are assembled.  Level 0 holds one
-// sum per (worker, tile); every higher level holds, per worker, the adjacent-pairs tree
-// sums of 64 consecutive nodes of the level below, up to a single root.  A node of level
-// L >= 1 also has an arrival counter: whoever delivers the last live child of a node sums
-// its children (in the fixed tree order, so the value does not depend on who does it),
-// resets the counter and delivers the node to its own parent.  Nobody waits for anybody.
-// The root of worker i is norm2[i]; whoever completes the last worker copies the K
-// results (and the status word) to pinned host memory and, when asked, runs the
-// weighting rule on them.  All counters are zero between rounds.
+// Where the squared distances ||x_i - c||^2 of a round are assembled.  A kernel that
+// measures distances only stores one sum per (worker, tile): level 0 of a tree in which
+// every higher level holds, per worker, the adjacent-pairs tree sums of 64 consecutive
+// nodes of the level below, up to a single root, norm2[i].  The upper levels are formed at
+// the head of the launch that needs the distances (the fused exchange that follows, or a
+// small kernel of its own for every other reader): the first `sync_ctas` CTAs share the
+// nodes of the large levels and meet at one arrival counter per level; levels with few
+// inputs are summed by every CTA for itself.  A CTA that has waited `wait_polls` polls for
+// the others sums the whole level itself, so nothing depends on the CTAs running at the
+// same time; the values are the same whoever forms them (fixed tree order).  CTA 0 also
+// copies the K results (and the status word) to pinned host memory and, when the rule is
+// asked for, stores the coefficients and the advanced history ring.  Level 0 has two
+// copies, so that a launch may assemble one round's sums while it stores the next one's.
+// The arrival counters only ever grow: a launch is told the value they reach with it.
 constexpr int kTreeRadixLog2 = 6;
 constexpr int kTreeMaxLevels = 4;      // 2^21 tiles at most (P < 2^31, 1024 parameters a tile)
+constexpr uint32_t kTreeOwnLevelInputs = 1024;   // a level with at most this many inputs (all
+                                                 // workers) is summed by every CTA for itself
 struct DistTree {
-    double *level0;                    // [K][n[0]], n[0] = tiles rounded up to a power of two
+    double *sums_out;                  // level 0 this launch stores: [K][n[0]], n[0] = tiles
+                                       //   rounded up to a power of two
+    const double *sums_in;             // level 0 this launch assembles (assemble != 0)
     double *upper;                     // level L >= 1: upper + K * off[L] + i * n[L] + node
-    uint32_t *count;                   // same indexing as upper
-    uint32_t *rows_done;               // workers whose root is complete this round
+    uint32_t *arrive;                  // [L]: CTAs that have delivered their share of level L
     double *norm2;                     // [K] roots
     double *norm2_host;                // pinned, mapped: [0] status word, [1 .. K] roots
     const uint32_t *status;            // device status word
-    RuleConfig rule;                   // the rule at the end of the round: its parameters,
-    double *uhist;                     //   the history ring [K][p + 1] on the device,
-    uint32_t *ring_flag;               //   whether the ring has been filled,
+    RuleConfig rule;                   // the weighting rule after the assembly: its parameters,
+    const double *ring_in;             //   the history ring [K][p + 1] it reads,
+    double *ring_out;                  //   the advanced ring it writes (another buffer),
     float *weights;                    //   and where the coefficients go: h2[K] then h1[K]
     double rule_alpha;
-    uint32_t run_rule;                 // 1: run the rule once every root is complete
+    uint32_t ring_filled;              // 0: the ring holds no sample yet
+    uint32_t run_rule;                 // 1: run the rule on the assembled distances
+    uint32_t assemble;                 // 1: this launch assembles sums_in at its head
+    uint32_t sync_ctas;                // CTAs 0 .. sync_ctas-1 share the large levels
+    uint32_t arrive_target;            // what arrive[L] reaches when they all have delivered
+    uint32_t wait_polls;               // polls before a CTA stops waiting for the others
+    uint32_t shared_levels;            // levels 1 .. shared_levels are the large ones
     uint32_t K;
     uint32_t levels;                   // level `levels` is the root (n == 1)
     uint32_t n[kTreeMaxLevels + 1];    // nodes per worker at each level

@@ -1,10 +1,12 @@
 // The smaller CUDA kernels (sm_100a) of the AdaHessian + elastic-averaging round: the
 // weighted elastic exchange, the Rademacher sampler for callers, the broadcast of the
-// master; and the entry to the fused local step, whose instantiations live in
+// master, the assembly of the distances for readers other than a fused exchange; and
+// the entry to the fused local step, whose instantiations live in
 // ah_step_inst.cu.  All HBM-bound streaming work: wide coalesced accesses, enough bytes
 // in flight, no byte touched twice.
 #include "ah_internal.h"
 #include "ah_device.cuh"
+#include "ah_tree.cuh"
 
 namespace ah {
 
@@ -81,9 +83,27 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
     st_vec(x + (uint64_t)blockIdx.y * lds + 4ull * q, ld_vec(c + 4ull * q));
 }
 
+// The distances ||x_i - c||^2 from the tile sums of the last distance round (and the
+// weighting rule on them, if it is owed), for the host, a snapshot or an exchange kernel:
+// T.sync_ctas CTAs of four warps.
+constexpr int kAssembleThreads = 128;
+__global__ void __launch_bounds__(kAssembleThreads)
+assemble_kernel(const __grid_constant__ DistTree T)
+{
+    __shared__ uint32_t word;
+    assemble_distances(T, (int)threadIdx.x, kAssembleThreads, blockIdx.x, nullptr, nullptr, &word,
+                       [] { __syncthreads(); });
+}
+
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
+cudaError_t launch_assemble(const DistTree &T, cudaStream_t s)
+{
+    assemble_kernel<<<T.sync_ctas, kAssembleThreads, 0, s>>>(T);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_step_inst_0(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);
 cudaError_t launch_step_inst_1(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);
 cudaError_t launch_step_inst_2(const StepParams &p, bool want_dist, int sm_count, cudaStream_t s);

@@ -247,10 +247,15 @@ __device__ __forceinline__ float4 apply_signs(float4 h, uint32_t nib)
 //
 // DIST additionally forms, per item, the pairwise-tree sum of (x_new - c)^2: the
 // consumer warps leave their eight partial sums in the stage, and the producer, when it
-// takes the stage back, adds them up and delivers the tile's sum to the arrival tree of
-// ah_tree.cuh, which ends in the K distances (and, if asked, the weighting rule) without
-// a launch of its own.  A worker that sits the step out contributes its unchanged x
+// takes the stage back, adds them up and stores the tile's sum (level 0 of the distance
+// tree of ah_tree.cuh).  A worker that sits the step out contributes its unchanged x
 // (only x and c are fetched for it).
+//
+// A fused exchange whose coefficients come from the weighting rule assembles the
+// distances of the preceding distance round from those tile sums at its head and runs
+// the rule there (the consumer warps of every CTA, while the producer already fetches the
+// first tiles): no launch, no copy and no host round trip lies between measuring the
+// distances and using the coefficients.
 //
 // The kernel may be launched with programmatic stream serialisation: everything before
 // griddepcontrol.wait touches only this CTA's shared memory and the launch parameters;
@@ -275,9 +280,7 @@ struct __align__(16) ItemHeader {
     uint32_t worker, t0, nvalid, flags;
     uint32_t e0, e1, run0, ea0;
     float bc1, bc2, rbc1, rbc2;            // the worker's bias corrections and reciprocals
-    uint32_t tile;
-    float h1, h2;                          // fused exchange: the worker's coefficients
-    uint32_t reserved;
+    uint32_t tile, reserved[3];
 };
 
 template <bool HASC>
@@ -304,6 +307,7 @@ struct __align__(128) Shared {
     uint64_t empty[kStages];               // consumers -> producer (stage drained)
     float h1[FUSE ? MAXW : 1];             // fused exchange: coefficients by worker index
     float h2[FUSE ? MAXW : 1];
+    uint32_t word;                         // fused exchange: scratch of the distance assembly
 };
 
 // All consumers learn whether every one of them saw the stage arrive.
@@ -440,53 +444,6 @@ __device__ __forceinline__ double stage_sum(const Stage<HASC> &st, int lane)
     return v;
 }
 
-// The producer's deliveries to the arrival tree, in batches of up to 32 so that the
-// memory round trips they need (a fence, the counters) are paid once per batch and never
-// hold up the next bulk copies.  Lane e of the producer owns entry e of a batch: it stores
-// the tile's sum at once (nobody waits for a store), and when the batch is full it fences
-// and counts its entry; what the counter returned is looked at when the next batch is
-// counted, or at the end.
-struct Deliveries {
-    uint32_t fill = 0;                      // entries of the batch being filled (same in every lane)
-    uint32_t my_i = 0, my_tile = 0;         // this lane's entry of that batch
-    uint32_t counted = 0;                   // entries of the batch whose counts are in flight
-    uint32_t c_i = 0, c_tile = 0, c_before = 0;   // this lane's entry of that batch
-
-    // the counts of the previous batch have come back: finish the nodes they completed
-    __device__ __forceinline__ void settle(const DistTree &T, int lane)
-    {
-        tree_after_counts(T, (uint32_t)lane < counted, c_i, c_tile, c_before, lane);
-        counted = 0;
-    }
-
-    // count the batch that has been filled
-    __device__ __forceinline__ void count(const DistTree &T, int lane)
-    {
-        settle(T, lane);
-        if ((uint32_t)lane < fill) c_before = tree_count_tile(T, my_i, my_tile);
-        c_i = my_i; c_tile = my_tile;
-        counted = fill;
-        fill = 0;
-    }
-
-    // a new tile sum (v in every lane)
-    __device__ __forceinline__ void add(const DistTree &T, uint32_t i, uint32_t tile, double v, int lane)
-    {
-        if ((uint32_t)lane == fill) {
-            tree_store_tile(T, i, tile, v);
-            my_i = i; my_tile = tile;
-        }
-        if (++fill == 32u) count(T, lane);
-    }
-
-    // nothing more comes: everything in flight is counted and settled
-    __device__ __forceinline__ void finish(const DistTree &T, int lane)
-    {
-        count(T, lane);
-        settle(T, lane);
-    }
-};
-
 // CTAs per SM an instantiation is built (register bound) and launched for.
 constexpr int ctas_per_sm(bool dist, bool multi, bool fuse)
 {
@@ -518,14 +475,6 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
 
     if (warp == kConsumerWarps) {
         // =============================== producer ===============================
-        if constexpr (FUSE) {
-            // exchange coefficients by worker index, from the device-side rule or the launch
-            for (uint32_t w = (uint32_t)lane; w < p.nworkers; w += 32u) {
-                sh.h1[w] = p.wdev ? p.wdev[p.nworkers + w] : p.h1w[w];
-                sh.h2[w] = p.wdev ? p.wdev[w] : p.h2w[w];
-            }
-            __syncwarp();
-        }
         // Items are drawn from the global counter one ahead of their use, so that the
         // round trip of the atomic overlaps the wait for a free stage.
         uint32_t drawn = 0;
@@ -533,7 +482,6 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
         uint32_t k = 0;
         uint32_t tile = 0, r = 0, rows_left = 0;   // FUSE: where the producer is in a tile's worker list
         bool healthy = true;
-        Deliveries deliveries;                     // DIST: tile sums on their way into the tree
         for (;; ++k) {
             const uint32_t s = k % kStages, use = k / kStages;
             Stage<HASC> &st = sh.stage[s];
@@ -542,8 +490,10 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                     healthy = false;
                     break;
                 }
-                if constexpr (DIST)                // the item that just left this stage
-                    deliveries.add(p.tree, st.hdr.worker, st.hdr.tile, stage_sum(st, lane), lane);
+                if constexpr (DIST) {              // the item that just left this stage
+                    const double sum = stage_sum(st, lane);
+                    if (lane == 0) tree_store_tile(p.tree, st.hdr.worker, st.hdr.tile, sum);
+                }
             }
             if (!FUSE || rows_left == 0u) {
                 const uint32_t n = __shfl_sync(0xffffffffu, drawn, 0);
@@ -598,9 +548,7 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                 const WorkerConst wc = p.w[i];
                 hd.bc1 = wc.bc1; hd.bc2 = wc.bc2; hd.rbc1 = wc.rbc1; hd.rbc2 = wc.rbc2;
                 hd.tile = tile;
-                hd.h1 = FUSE ? sh.h1[i] : 0.f;
-                hd.h2 = FUSE ? sh.h2[i] : 0.f;
-                hd.reserved = 0u;
+                hd.reserved[0] = hd.reserved[1] = hd.reserved[2] = 0u;
                 st.hdr = hd;
             }
             __syncwarp();
@@ -642,9 +590,9 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                 if (use == 0u) continue;
                 if (!mbar_wait(&sh.empty[s], (use - 1u) & 1u, p.status, kStatusEmptyTimeout)) break;
                 const Stage<HASC> &st = sh.stage[s];
-                deliveries.add(p.tree, st.hdr.worker, st.hdr.tile, stage_sum(st, lane), lane);
+                const double sum = stage_sum(st, lane);
+                if (lane == 0) tree_store_tile(p.tree, st.hdr.worker, st.hdr.tile, sum);
             }
-            deliveries.finish(p.tree, lane);
         }
         // the last producer to leave puts both scheduler words back to zero for the next
         // launch (every producer has made its final fetch before it counts itself out)
@@ -660,6 +608,20 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
 
     // ================================= consumers =================================
     const int ctid = threadIdx.x;
+    if constexpr (FUSE) {
+        // exchange coefficients by worker index: from the weighting rule, run here on the
+        // distances this launch assembles first, or from device memory, or from the launch
+        const bool rule_here = p.tree.assemble != 0u && p.tree.run_rule != 0u;
+        if (p.tree.assemble)
+            assemble_distances(p.tree, ctid, kConsumers, blockIdx.x, rule_here ? sh.h1 : nullptr,
+                               sh.h2, &sh.word, [] { consumer_sync(); });
+        if (!rule_here)
+            for (uint32_t w = (uint32_t)ctid; w < p.nworkers; w += (uint32_t)kConsumers) {
+                sh.h1[w] = p.wdev ? p.wdev[p.nworkers + w] : p.h1w[w];
+                sh.h2[w] = p.wdev ? p.wdev[w] : p.h2w[w];
+            }
+        consumer_sync();
+    }
     float4 c_old[kPasses], c_acc[kPasses];         // FUSE: carried through the workers of a tile
     uint32_t k = 0;
     for (;; ++k) {
@@ -680,8 +642,8 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
         const bool meets_first = meets && p.pull_first != 0u;
         float h1 = 0.f, h2 = 0.f;
         if constexpr (FUSE) {
-            h1 = st.hdr.h1;
-            h2 = st.hdr.h2;
+            h1 = sh.h1[i];
+            h2 = sh.h2[i];
             if (flags & kItemFirst) {
 #pragma unroll
                 for (int pass = 0; pass < kPasses; ++pass) {

@@ -92,17 +92,10 @@ sgd_step_kernel(const __grid_constant__ SgdParams p)
     }
     if (DIST) {
         __syncthreads();
-        if (warp == 0) {
-            // one warp delivers the CTA's tile sums to the arrival tree: lane k stores and
-            // counts tile k, then every lane whose count completed a node climbs with it
-            const bool mine = lane < kTilesPerCta && tile0 + lane < p.ntiles;
-            uint32_t before = 0;
-            if (mine) {
-                tree_store_tile(p.tree, i, tile0 + lane, tree8(red[lane]));
-                before = tree_count_tile(p.tree, i, tile0 + lane);
-            }
-            tree_after_counts(p.tree, mine, i, tile0 + lane, before, lane);
-        }
+        // the CTA's tile sums go to level 0 of the distance tree; whoever needs the
+        // distances assembles them
+        if (warp == 0 && lane < kTilesPerCta && tile0 + lane < p.ntiles)
+            tree_store_tile(p.tree, i, tile0 + lane, tree8(red[lane]));
     }
 }
 
@@ -237,11 +230,10 @@ extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const s
         step[i] = h->step[i] + (on ? 1u : 0u);
         if (on || dist) p.row[p.nrows++] = (uint16_t)i;   // distances cover every worker
     }
+    p.tree = h->tree;
     if (dist) {
-        const int rc = prepare_distance_round(h, false, 0.f, p.tree);
+        const int rc = begin_distance_store(h, p.tree);
         if (rc != AH_OK) return rc;
-    } else {
-        memset(&p.tree, 0, sizeof p.tree);
     }
     cudaError_t e;
     const bool mom = hy->momentum != 0.f;
@@ -251,7 +243,7 @@ extern "C" int sgd_local_step(ah_ctx *h, const float *grad, uint64_t ld, const s
     h->calls += 1;
     memcpy(h->step, step, (size_t)h->K * sizeof(uint32_t));
     if (p.nrows) h->launches += 1;
-    if (dist) return finish_distances(h);
+    if (dist && p.nrows) commit_distance_store(h, false, 0.f, false);
     return AH_OK;
 }
 

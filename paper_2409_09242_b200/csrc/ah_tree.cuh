@@ -1,10 +1,8 @@
-// Assembly of the squared distances ||x_i - c||^2 (Sec. V-B: u = log ||x_i - c||) inside
-// the kernels that produce the per-tile sums, with no launch of its own: an arrival tree
-// of radix 64 over the tiles of each worker (see DistTree), then, by whoever completes
-// the last worker, the copy of the results to pinned host memory and the weighting rule
-// of Sec. V-B (Eqs. 10-11, h1 / h2).  The sums follow the same adjacent-pairs binary tree
-// whatever the order of arrival, so the result is a pure function of the tile sums.
-// Not installed.
+// Assembly of the squared distances ||x_i - c||^2 (Sec. V-B: u = log ||x_i - c||) from
+// the per-tile sums that a distance round stores (see DistTree), at the head of the launch
+// that needs them, and the weighting rule of Sec. V-B (Eqs. 10-11, h1 / h2) on the result.
+// The sums follow the same adjacent-pairs binary tree whoever forms them, so the result
+// is a pure function of the tile sums.  Not installed.
 #pragma once
 
 #include "ah_device.cuh"
@@ -13,170 +11,143 @@
 
 namespace ah {
 
-// Orders this thread's earlier writes before its later ones, and its later reads after
-// its earlier ones, as seen from anywhere on the GPU (lighter than the sequentially
-// consistent __threadfence()).
+// Orders this thread's earlier writes (and those it has observed) before its later ones,
+// and its later reads after its earlier ones, as seen from anywhere on the GPU (lighter
+// than the sequentially consistent __threadfence()).
 __device__ __forceinline__ void fence_gpu()
 {
     asm volatile("fence.acq_rel.gpu;" ::: "memory");
 }
 
-// By one warp, after every root of the round is complete: results and status word to the
-// host copy, then the rule for all workers.  Kept out of line: it runs once per round and
-// its double-double logarithm would otherwise claim registers in the streaming kernels.
-static __device__ __noinline__ void finish_round(const DistTree &T, int lane)
+__device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t *p)
 {
-    fence_gpu();                                       // the roots other warps wrote
-    const bool filled = __ldcg(T.ring_flag) != 0u;
-    __syncwarp();
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// A distance round's only contribution: the tile's sum goes to its level-0 slot.
+__device__ __forceinline__ void tree_store_tile(const DistTree &T, uint32_t i, uint32_t tile, double v)
+{
+    T.sums_out[(size_t)i * T.n[0] + tile] = v;
+}
+
+// Nodes first, first + stride, ... of level L (numbered worker by worker over the live
+// nodes), each by one warp: two children a lane, then the butterfly (the adjacent-pairs
+// order).  Four nodes' loads are in flight before the first sum is formed.
+__device__ __forceinline__ void tree_sum_nodes(const DistTree &T, uint32_t L, uint32_t first,
+                                               uint32_t stride, int lane)
+{
+    const uint32_t per = T.live[L], total = T.K * per;
+    const double *below = L == 1u ? T.sums_in : T.upper + (size_t)T.K * T.off[L - 1u];
+    const uint32_t below_n = T.n[L - 1u], below_live = T.live[L - 1u];
+    for (uint32_t base = first; base < total; base += 4u * stride) {
+        double pair[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t node = base + (uint32_t)q * stride;
+            pair[q] = 0.0;
+            if (node < total) {
+                const uint32_t i = node / per, nd = node - i * per;
+                const uint32_t children = min(1u << kTreeRadixLog2, below_live - (nd << kTreeRadixLog2));
+                const double *child = below + (size_t)i * below_n + ((size_t)nd << kTreeRadixLog2);
+                const uint32_t a = 2u * (uint32_t)lane, b = a + 1u;
+                const double va = a < children ? __ldcg(child + a) : 0.0;
+                const double vb = b < children ? __ldcg(child + b) : 0.0;
+                pair[q] = __dadd_rn(va, vb);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t node = base + (uint32_t)q * stride;
+            if (node < total) {                            // the same for every lane
+                const double sum = warp_tree_sum(pair[q]);
+                if (lane == 0) {
+                    const uint32_t i = node / per, nd = node - i * per;
+                    if (L == T.levels) T.norm2[i] = sum;
+                    else T.upper[(size_t)T.K * T.off[L] + (size_t)i * T.n[L] + nd] = sum;
+                }
+            }
+        }
+    }
+}
+
+// The whole assembly, by `nthreads` threads (whole warps) of every CTA of the launch;
+// `sync` is a barrier over exactly those threads and `scratch` one word of shared memory.
+// Afterwards every calling CTA may read norm2[0 .. K) (with __ldcg), and, if the rule was
+// asked for, finds the coefficients of worker w in h1s[w], h2s[w] (shared memory, may be
+// null).  Kept out of line: it runs once per launch, and its double-double logarithm
+// would otherwise claim registers in the streaming kernels.
+template <class Sync>
+static __device__ __noinline__ void assemble_distances(const DistTree &T, int tid, int nthreads,
+                                                       uint32_t cta, float *h1s, float *h2s,
+                                                       uint32_t *scratch, Sync sync)
+{
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
+    for (uint32_t L = 1u; L <= T.levels; ++L) {
+        if (L > T.shared_levels) {
+            // few inputs: every CTA forms the whole level for itself (the CTAs store the
+            // same values to the same places)
+            tree_sum_nodes(T, L, (uint32_t)warp, (uint32_t)nwarps, lane);
+            sync();
+            continue;
+        }
+        if (cta < T.sync_ctas)
+            tree_sum_nodes(T, L, cta * (uint32_t)nwarps + (uint32_t)warp,
+                           T.sync_ctas * (uint32_t)nwarps, lane);
+        sync();                                            // this CTA's share is stored
+        if (tid == 0) {
+            if (cta < T.sync_ctas) {
+                fence_gpu();                               // ... and visible before it is counted
+                atomicAdd(&T.arrive[L], 1u);
+            }
+            uint32_t polls = 0;
+            bool there;
+            while (!(there = (int32_t)(ld_relaxed_gpu(&T.arrive[L]) - T.arrive_target) >= 0) &&
+                   polls < T.wait_polls) {
+                ++polls;
+                __nanosleep(64);
+            }
+            fence_gpu();                                   // what the counter announced is visible
+            *scratch = there ? 0u : 1u;
+        }
+        sync();
+        const bool alone = *scratch != 0u;
+        sync();                                            // the word may be written again
+        if (alone) {                                       // the others are late: the whole level here
+            tree_sum_nodes(T, L, (uint32_t)warp, (uint32_t)nwarps, lane);
+            sync();
+        }
+    }
+    // ---- results to the host copy, the rule
     WeightRule rule;
+    const size_t depth = (size_t)T.rule.p_hist + 1u;
     if (T.run_rule) {
         rule.p_hist = T.rule.p_hist;
         for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = T.rule.coef[j];
         rule.kappa = T.rule.kappa;
         rule.alpha = T.rule_alpha;
     }
-    for (uint32_t w = (uint32_t)lane; w < T.K; w += 32u) {
+    for (uint32_t w = (uint32_t)tid; w < T.K; w += (uint32_t)nthreads) {
         const double n2 = __ldcg(&T.norm2[w]);
-        T.norm2_host[1u + w] = n2;
-        if (T.run_rule)
-            weight_rule_step(rule, n2, T.uhist + (size_t)w * (size_t)(rule.p_hist + 1), filled,
-                             &T.weights[w], &T.weights[T.K + w]);
+        if (cta == 0u) T.norm2_host[1u + w] = n2;
+        if (T.run_rule) {
+            float to_master, to_worker;
+            weight_rule_step(rule, n2, T.ring_in + (size_t)w * depth,
+                             cta == 0u ? T.ring_out + (size_t)w * depth : nullptr,
+                             T.ring_filled != 0u, &to_master, &to_worker);
+            if (h1s) { h1s[w] = to_worker; h2s[w] = to_master; }
+            if (cta == 0u) { T.weights[w] = to_master; T.weights[T.K + w] = to_worker; }
+        }
     }
-    if (lane == 0) {
+    if (cta == 0u && tid == 0) {
         // the status word travels as the bit pattern of the first double, as it sits in
-        // device memory in front of the distances
+        // device memory in front of the distances; the host reads its copy only behind an
+        // event that follows this kernel
         reinterpret_cast<uint32_t *>(T.norm2_host)[0] = __ldcg(T.status);
         reinterpret_cast<uint32_t *>(T.norm2_host)[1] = 0u;
-        if (T.run_rule) *T.ring_flag = 1u;
     }
-    // the host reads its copy only behind an event that follows this kernel
-}
-
-// Live children of node `parent` of level L (L >= 1): nodes of level L - 1 that exist.
-__device__ __forceinline__ uint32_t tree_children(const DistTree &T, uint32_t L, uint32_t parent)
-{
-    return min(1u << kTreeRadixLog2, T.live[L - 1] - (parent << kTreeRadixLog2));
-}
-
-__device__ __forceinline__ uint32_t *tree_counter(const DistTree &T, uint32_t L, uint32_t i,
-                                                  uint32_t node)
-{
-    return T.count + (size_t)T.K * T.off[L] + (size_t)i * T.n[L] + node;
-}
-
-// A tile's sum reaches the tree in three steps that a caller may spread over time, so
-// that no memory round trip sits on its critical path (each step by itself is correct
-// however long after the previous one it runs):
-//   1. tree_store_tile  (one lane)   the sum goes to its level-0 slot;
-//   2. tree_count_tile  (same lane)  a fence, then the arrival is counted at the tile's
-//                                    level-1 node; returns the arrivals before this one;
-//   3. tree_after_counts (whole warp, one counted tile per lane) where an arrival was its
-//                                    node's last, the node is summed and delivered upwards,
-//                                    as far as that completes nodes.
-__device__ __forceinline__ void tree_store_tile(const DistTree &T, uint32_t i, uint32_t tile, double v)
-{
-    T.level0[(size_t)i * T.n[0] + tile] = v;
-}
-
-__device__ __forceinline__ uint32_t tree_count_tile(const DistTree &T, uint32_t i, uint32_t tile)
-{
-    fence_gpu();                                       // the sum is visible before it is counted
-    return atomicAdd(tree_counter(T, 1u, i, tile >> kTreeRadixLog2), 1u);
-}
-
-// Every lane with `climbing` set has just completed the level-1 node above its tile.  The
-// warp sums those nodes one after the other, all 32 lanes on one node at a time (two
-// children a lane, then the butterfly: the adjacent-pairs order; the loads of eight nodes
-// are issued before the first sum is formed), delivers each to its parent, and repeats
-// with the lanes whose delivery completed the parent.  All 32 lanes must call; at the
-// top, whoever completes the last worker has the whole warp finish the round.
-static __device__ __noinline__ void tree_climb(const DistTree &T, bool climbing, uint32_t i,
-                                               uint32_t tile, int lane)
-{
-    uint32_t node = tile >> kTreeRadixLog2, L = 1u;
-    bool last_row = false;
-    fence_gpu();                                       // counted children are visible from here on
-    for (uint32_t todo = __ballot_sync(0xffffffffu, climbing); todo != 0u;
-         todo = __ballot_sync(0xffffffffu, climbing)) {
-        // the nodes of this pass, eight at a time: loads first, sums after
-        double mine = 0.0;                             // lane e ends up with the sum of its own node
-        for (uint32_t rest = todo; rest != 0u;) {
-            double pair[8];
-            int owner[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                owner[q] = rest ? __ffs(rest) - 1 : -1;
-                if (rest) rest &= rest - 1u;
-                pair[q] = 0.0;
-                if (owner[q] >= 0) {
-                    const uint32_t oi = __shfl_sync(0xffffffffu, i, owner[q]);
-                    const uint32_t on = __shfl_sync(0xffffffffu, node, owner[q]);
-                    const uint32_t oL = __shfl_sync(0xffffffffu, L, owner[q]);
-                    const double *below = oL == 1u ? T.level0 + (size_t)oi * T.n[0]
-                                                   : T.upper + (size_t)T.K * T.off[oL - 1u] + (size_t)oi * T.n[oL - 1u];
-                    const uint32_t children = tree_children(T, oL, on);
-                    const double *child = below + ((size_t)on << kTreeRadixLog2);
-                    const uint32_t a = 2u * (uint32_t)lane, b = a + 1u;
-                    const double va = a < children ? __ldcg(child + a) : 0.0;
-                    const double vb = b < children ? __ldcg(child + b) : 0.0;
-                    pair[q] = __dadd_rn(va, vb);
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                if (owner[q] >= 0) {
-                    const double sum = warp_tree_sum(pair[q]);
-                    if (lane == owner[q]) mine = sum;
-                }
-        }
-        // every owner delivers its node upwards
-        if (climbing) {
-            *tree_counter(T, L, i, node) = 0u;         // ready for the next round
-            if (L == T.levels) {                       // the root of worker i
-                T.norm2[i] = mine;
-                fence_gpu();
-                last_row = atomicAdd(T.rows_done, 1u) + 1u == T.K;
-                climbing = false;
-            } else {
-                T.upper[(size_t)T.K * T.off[L] + (size_t)i * T.n[L] + node] = mine;
-                fence_gpu();
-                const uint32_t parent = node >> kTreeRadixLog2;
-                climbing = atomicAdd(tree_counter(T, L + 1u, i, parent), 1u) + 1u ==
-                           tree_children(T, L + 1u, parent);
-                node = parent;
-                ++L;
-            }
-        }
-        fence_gpu();                                   // what the counters announced is visible
-    }
-    if (__any_sync(0xffffffffu, last_row)) {
-        if (last_row) *T.rows_done = 0u;
-        finish_round(T, lane);
-    }
-}
-
-// Step 3 for a whole warp at once: lane by lane, (valid, i, tile, before) describe one
-// counted tile sum.  All 32 lanes, converged.  The common case (no count completed a
-// node) costs one vote.
-__device__ __forceinline__ void tree_after_counts(const DistTree &T, bool valid, uint32_t i,
-                                                  uint32_t tile, uint32_t before, int lane)
-{
-    const bool climbing = valid && before + 1u == tree_children(T, 1u, tile >> kTreeRadixLog2);
-    if (__any_sync(0xffffffffu, climbing)) tree_climb(T, climbing, i, tile, lane);
-}
-
-// The three steps at once for one tile sum.  All 32 lanes of a converged warp; `value`
-// counts in lane 0.
-__device__ __forceinline__ void deliver_tile_sum(const DistTree &T, uint32_t i, uint32_t tile,
-                                                 double value, int lane)
-{
-    uint32_t before = 0;
-    if (lane == 0) {
-        tree_store_tile(T, i, tile, value);
-        before = tree_count_tile(T, i, tile);
-    }
-    tree_after_counts(T, lane == 0, i, tile, before, lane);
+    sync();
 }
 
 }  // namespace ah

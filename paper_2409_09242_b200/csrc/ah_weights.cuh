@@ -17,14 +17,17 @@ struct WeightRule {
 
 // Pushes the sample u = log ||x_i - c|| into the worker's ring (newest first; the
 // first sample fills the whole ring), forms the raw score of Eqs. 10-11 and maps it
-// through h1 (worker-side coefficient) and h2 (master-side coefficient).
-__host__ __device__ inline void weight_rule_step(const WeightRule &rule, double norm2, double *ring,
+// through h1 (worker-side coefficient) and h2 (master-side coefficient).  The ring is read
+// from ring_in and the advanced ring goes to ring_out (the same array, another one, or
+// null where somebody else stores it).
+__host__ __device__ inline void weight_rule_step(const WeightRule &rule, double norm2,
+                                                 const double *ring_in, double *ring_out,
                                                  bool ring_filled, float *to_master, float *to_worker)
 {
     // the ring is read in one go (the loads do not wait for one another), moved on in
     // registers and written back at the end
     double past[AH_MAX_HIST + 1];
-    for (int j = 0; j <= rule.p_hist; ++j) past[j] = ring[j];
+    for (int j = 0; j <= rule.p_hist; ++j) past[j] = ring_in[j];
     const double u = u_from_norm2(norm2);
     if (ring_filled) {
         for (int j = rule.p_hist; j >= 1; --j) past[j] = past[j - 1];
@@ -35,7 +38,8 @@ __host__ __device__ inline void weight_rule_step(const WeightRule &rule, double 
     double score = 0.0;
     for (int j = 0; j < rule.p_hist; ++j)
         score = AH_DADD(score, AH_DMUL(rule.coef[j], AH_DSUB(past[j], past[j + 1])));
-    for (int j = 0; j <= rule.p_hist; ++j) ring[j] = past[j];
+    if (ring_out)
+        for (int j = 0; j <= rule.p_hist; ++j) ring_out[j] = past[j];
     double w_worker, w_master;
     if (score < rule.kappa) {
         w_worker = 1.0;

@@ -40,6 +40,8 @@ class RunConfig:
     scripted: list = field(default_factory=list)
     pool: int = 3
     data_seed: int = 0
+    wait_polls: int | None = None   # library setting: how long the CTAs that assemble the
+                                    # distances wait for one another (0: each works alone)
 
     def alpha_value(self):
         return min(0.05, 0.8 / self.K) if self.alpha is None else self.alpha
@@ -63,6 +65,8 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
     h = binding.Handle(cfg.K, cfg.P, cfg.segments)
     h.ah_state_set(binding.AH_CENTER, theta0)
     h.ah_broadcast_center()
+    if cfg.wait_polls is not None:
+        h.ah_set_wait_polls(cfg.wait_polls)
     ref = oracle_mod.OracleState(theta0, cfg.K, cfg.segments, variant=variant)
     alpha = cfg.alpha_value()
     log = {"weights_equal": True, "masks_equal": True, "norm2_equal": True, "orders_equal": True,
@@ -83,7 +87,7 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
             # the library defers each exchange to the local step of the following round; the
             # oracle exchanges at once.  States agree whenever no exchange is pending.
             if pending is not None:
-                p_mask, p_order, p_h2, p_h1 = pending
+                p_mask, p_order, p_h2, p_h1, p_norm2 = pending
                 h.easgd_exchange_then_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
                                            active=mask_g if cfg.frozen else None, worker_mask=p_mask,
                                            alpha=alpha, order=p_order, asynchronous=cfg.asynchronous,
@@ -93,12 +97,14 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                     w = h.ah_state_get(binding.AH_WEIGHTS)
                     log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], p_h2) and
                                                  np.array_equal(w[cfg.K:], p_h1))
+                if p_norm2 is not None:      # assembled at the head of the riding launch
+                    log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), p_norm2))
                 pending = None
                 assert not ex, "tau >= 2"
             else:
-                # every other distance round also runs the weighting rule in its last kernel
-                # (AH_DIST_AND_RULE, the shape the benchmark times); the others leave it to
-                # the call that makes the exchange
+                # every other distance round also asks for the weighting rule (AH_DIST_AND_RULE,
+                # the shape the benchmark times); the others leave that to the call that makes
+                # the exchange
                 rule_now = ex and cfg.dynamic and log["exchanges"] % 2 == 0
                 h.ah_local_step(dev_pool[k][0], dev_pool[k][1], Z_SEED, round_=t,
                                 active=mask_g if cfg.frozen else None,
@@ -108,7 +114,11 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                            active=mask_o if cfg.frozen else None, **common)
             if ex:
                 log["exchanges"] += 1
-                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+                # Reading the distances now has them assembled by a kernel of their own; left
+                # alone, the riding launch assembles them at its head.  Both ways are taken.
+                look_now = log["exchanges"] % 3 == 0 or t == cfg.rounds
+                if look_now:
+                    log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
                 order_g = order_o = None
                 if cfg.asynchronous:
                     order_g = h.dw_order_next(ORDER_SEED, t)
@@ -119,7 +129,7 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                     ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
                 else:
                     ref.exchange(mask_o, h2, h1, alpha=alpha)
-                pending = (mask_g, order_g, h2, h1)
+                pending = (mask_g, order_g, h2, h1, None if look_now else ref.norm2.copy())
                 if t == cfg.rounds:                                  # nothing follows: exchange now
                     if cfg.dynamic:
                         h.easgd_exchange_dynamic(mask_g, alpha, order_g, cfg.asynchronous)
@@ -149,15 +159,21 @@ def run_gaussian(cfg: RunConfig, binding, oracle_mod, layout_inputs, variant="om
                 ref.exchange_async(mask_o, h2, h1, alpha=alpha, order=order_o)
             else:
                 ref.exchange(mask_o, h2, h1, alpha=alpha)
-            log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
+            # Looking at the distances or the coefficients now has them assembled by a kernel
+            # of their own; left alone, the next lagged round does it at its head (what it
+            # used then shows in the state).  Both ways are taken.
+            look_now = not lag or log["exchanges"] % 2 == 0 or t + cfg.tau > cfg.rounds
+            if look_now:
+                log["norm2_equal"] &= bool(np.array_equal(h.ah_state_get(binding.AH_NORM2), ref.norm2))
             if lag:
                 lagged_weights = ref.weights_next(alpha)            # serves the next exchange round
-                w = h.ah_state_get(binding.AH_WEIGHTS)
-                log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], lagged_weights[0]) and
-                                             np.array_equal(w[cfg.K:], lagged_weights[1]))
+                if look_now:
+                    w = h.ah_state_get(binding.AH_WEIGHTS)
+                    log["weights_equal"] &= bool(np.array_equal(w[:cfg.K], lagged_weights[0]) and
+                                                 np.array_equal(w[cfg.K:], lagged_weights[1]))
             continue
-        # where the weights of this exchange come from: the device (the rule either in the
-        # last kernel of the distance round or as a launch of its own) or the host
+        # where the weights of this exchange come from: the device (the rule either owed by
+        # the distance round or asked for by the exchange) or the host
         ex_index = log["exchanges"] + 1
         on_device = ex and cfg.dynamic and (cfg.sync_free == "yes" or
                                             (cfg.sync_free == "mixed" and ex_index % 2 == 1))

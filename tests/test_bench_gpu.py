@@ -35,7 +35,8 @@ def test_bench_line_on_the_small_profiling_case():
     assert r["algorithmic_bytes_per_launch"] == 32 * 4 * 11_689_512
     assert r["launches_bracketed"] >= 10 and r["ms_per_launch"] > 0
     # one period is four launches: the exchange riding on the first step, two plain steps and a
-    # distance round whose last kernel also sums the distances and runs the weighting rule
+    # distance round that stores its tile sums (the riding exchange of the next period assembles
+    # the distances and runs the weighting rule at its head)
     assert line["gpu_launches"] == 4 * line["steps"] * line["reps"]
     e = line["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0

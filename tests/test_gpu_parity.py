@@ -333,9 +333,9 @@ def test_async_rounds_resnet18_shape_reduced(B, torch):
 
 @pytest.mark.parametrize("K,width", [(40, 16), (256, 16)])
 def test_many_workers_with_the_rule_inside_the_distance_round(B, torch, K, width):
-    # more workers than lanes in a warp (the rule takes several workers per lane), the large
-    # per-worker launch tables, distances and rule inside the step kernel, the exchange riding on
-    # the next step: the shape the benchmark times for its largest worker counts
+    # more workers than consumer threads in a CTA (the rule takes several workers per thread), the
+    # large per-worker launch tables, distances assembled and rule run at the head of the riding
+    # exchange: the shape the benchmark times for its largest worker counts
     layout = W.resnet18_layout(width)
     cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=12, tau=2,
                     p_fail=0.2, max_stale=3, frozen=True, fused="next")
@@ -346,6 +346,55 @@ def test_many_workers_with_the_rule_inside_the_distance_round(B, torch, K, width
     assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
     assert log["exchanges"] == 6
     h.close()
+
+
+@pytest.mark.parametrize("polls,K,width", [(0, 8, 8), (1, 8, 8), (0, 40, 16), (0, 4, 32)])
+def test_assembly_when_the_ctas_do_not_wait_for_one_another(B, torch, polls, K, width):
+    # wait budget 0 (or one poll): every CTA of a launch that assembles the distances gives up on
+    # the others at once and forms the whole tree by itself; same tree, same bits
+    layout = W.resnet18_layout(width)
+    cfg = RunConfig(K=K, segments=W.segments(layout), P=W.total_params(layout), rounds=24, tau=2,
+                    p_fail=0.25, fused="next", wait_polls=polls)
+    h, ref, log = run_gaussian(cfg, B, oracle, _layout_inputs(layout, K, n_pool=2), variant="omp")
+    viol, bits = compare_state(h, ref, B)
+    assert log["masks_equal"] and log["weights_equal"] and log["norm2_equal"], log
+    assert sum(viol.values()) == 0 and sum(bits.values()) == 0, (viol, bits)
+    assert np.array_equal(h.ah_state_get(B.AH_UHIST), ref.uhist)
+    assert log["exchanges"] == 12
+    h.close()
+
+
+def test_riding_exchange_assembles_the_distances_without_a_launch_of_its_own(B, torch):
+    # distance round, then the exchange riding on the next step: two launches, and the riding
+    # one leaves the distances where a reader finds them; a twin that reads them at once (a
+    # kernel of their own assembles them) sees the same bits and ends in the same state
+    K, P = 4, 300_001
+    rng = np.random.default_rng(7)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    ld = W.padded_ld(P)
+    g = torch.from_numpy(rng.standard_normal((K, ld)).astype(np.float32)).cuda()
+    hv = torch.from_numpy(rng.standard_normal((K, ld)).astype(np.float32)).cuda()
+    mask = np.ones(K, np.uint8)
+    seen = []
+    for read_at_once in (False, True):
+        h = B.Handle(K, P, [])
+        h.ah_state_set(B.AH_CENTER, theta0)
+        h.ah_broadcast_center()
+        n0 = h.ah_launch_count()
+        h.ah_local_step(g, hv, 1, round_=1, lr=0.01, want_dist=B.AH_DIST_AND_RULE, rule_alpha=0.05)
+        first = h.ah_state_get(B.AH_NORM2).copy() if read_at_once else None
+        h.easgd_exchange_then_step(g, hv, 1, round_=2, lr=0.01, worker_mask=mask, alpha=0.05, dynamic=True)
+        assert h.ah_launch_count() - n0 == (3 if read_at_once else 2)
+        n2 = h.ah_state_get(B.AH_NORM2).copy()
+        assert h.ah_launch_count() - n0 == (3 if read_at_once else 2)
+        if read_at_once:
+            assert np.array_equal(first, n2)
+        seen.append((n2, h.ah_state_get(B.AH_WEIGHTS).copy(), h.ah_state_get(B.AH_X).copy(),
+                     h.ah_state_get(B.AH_CENTER).copy(), h.ah_state_get(B.AH_UHIST).copy()))
+        h.close()
+    for a, b in zip(*seen):
+        assert np.array_equal(a, b)
+    assert np.all(seen[0][0] > 0)
 
 
 # --------------------------------------- weights on the device, no host round trip
@@ -931,8 +980,8 @@ def test_checkpoint_resume_with_the_rule_on_the_device(B, torch):
 def test_checkpoint_resume_with_an_exchange_pending(B, torch):
     # the bench's default shape: the exchange of a period rides on the first local step of the
     # next one, so at a period boundary something waits on the device: the distances (the rule
-    # still to run), or the coefficients the rule made of them at the end of the distance
-    # round.  A snapshot taken there, restored into a fresh handle, must continue bit for bit:
+    # still to run), or the coefficients of a rule the distance round asked for (the snapshot
+    # has them assembled and the rule run).  A snapshot taken there, restored into a fresh handle, must continue bit for bit:
     # in the first case the restored distances are pending again, in the second the restored
     # coefficients are handed to the exchange as caller weights.
     layout = W.resnet18_layout(16)
@@ -1047,7 +1096,7 @@ def test_error_paths_and_own_allocation(B, torch):
     # the handle still works after the refusals
     h.ah_local_step(g, g, 1, lr=0.01, want_dist=True)
     assert np.all(h.dw_weights_next(0.1) == np.float32(0.1))
-    assert h.ah_launch_count() == 1                  # the distances cost no launch of their own
+    assert h.ah_launch_count() == 2                  # the step, and the assembly of its tile sums for the host
     # a refused call changes nothing: step counts and the call counter stay where they were
     steps, calls = h.ah_state_get(B.AH_STEP).copy(), h.ah_state_get(B.AH_ROUND).copy()
     assert lib.ah_local_step(h._h, g.data_ptr(), g.data_ptr(), 1002, 1, C.byref(hy)) == B.AH_ERR_ALIGN
@@ -1060,7 +1109,7 @@ def test_error_paths_and_own_allocation(B, torch):
                                         0.1, None, 0, 1) == B.AH_ERR_STATE  # no distances pending
     assert np.array_equal(h.ah_state_get(B.AH_STEP), steps)
     assert np.array_equal(h.ah_state_get(B.AH_ROUND), calls)
-    assert h.ah_launch_count() == 1
+    assert h.ah_launch_count() == 2
     h.close()
     # a workspace that is too small is refused
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")
