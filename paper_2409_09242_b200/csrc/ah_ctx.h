@@ -27,8 +27,8 @@ struct ah_ctx {
     double *sums[2] = {nullptr, nullptr};   // level 0 of the distance tree, two copies: [K][ntiles_pad]
     int sums_cur = 0;              // the copy that holds the latest distance round's tile sums
     ah::DistTree tree;             // the tree's shape and fixed addresses (per-launch fields unset)
-    uint32_t arrive_total = 0;     // what the tree's arrival counters stand at
-    bool tree_dirty = false;       // a kernel gave up half way: clear the arrival counters first
+    uint32_t arrive_total[ah::kTreeMaxLevels + 1] = {};   // what the tree's counters stand at
+    bool tree_dirty = false;       // a kernel gave up half way: clear the tree's counters first
     uint32_t wait_polls = 4096;    // how long the CTAs of an assembling launch wait for one another
     double *norm2_dev = nullptr;   // [0] holds the status word, [1..K] the distances
     uint32_t *sched = nullptr;     // item scheduler of the local-step kernel (2 words)
@@ -81,7 +81,7 @@ namespace ah {
 // ah_host.cu: the life of a distance round's tile sums
 int begin_distance_store(ah_ctx *h, DistTree &tree);       // a launch is about to store a round's sums
 void commit_distance_store(ah_ctx *h, bool rule, float alpha, bool owed_to_exchange);
-int begin_assembly(ah_ctx *h, bool run_rule, float alpha, uint32_t sync_ctas, DistTree &tree);
+int begin_assembly(ah_ctx *h, bool run_rule, float alpha, DistTree &tree);
 int commit_assembly(ah_ctx *h, const DistTree &tree);
 int settle_distances(ah_ctx *h);   // assembles waiting sums with a kernel of its own, if any
 int ring_to_host(ah_ctx *h);
@@ -90,5 +90,5 @@ int enqueue_weight_rule(ah_ctx *h, float alpha);   // ah_dynamic.cu
 int fill_exchange(ah_ctx *h, const uint8_t *worker_mask, const float *weights, float alpha,
                   const uint16_t *order, const float *weights_dev, ExchangeParams &p);
 cudaError_t launch_exchange_in_order(const ExchangeParams &p, cudaStream_t s);   // ah_exchange_async.cu
-cudaError_t launch_assemble(const DistTree &T, cudaStream_t s);                  // ah_kernels.cu
+cudaError_t launch_assemble(const DistTree &T, uint32_t ctas, cudaStream_t s);   // ah_kernels.cu
 }

@@ -2,6 +2,8 @@
 // computed on the device from the distances the preceding local step left there, and
 // the exchange kernel reads them from device memory.  The host never waits, so the
 // next period's launches can be queued while this one still runs.
+#include <string.h>
+
 #include "ah_ctx.h"
 #include "ah_weights.cuh"
 
@@ -10,13 +12,14 @@ namespace ah {
 // One thread per worker: the weighting rule for worker i (the same function the host
 // entry points run), on the device copy of the history ring.
 __global__ void __launch_bounds__(AH_MAX_WORKERS)
-dynamic_weights_kernel(const __grid_constant__ WeightRule rule, const double *norm2, double *uhist,
-                       bool filled, float *weights, int nworkers)
+dynamic_weights_kernel(const __grid_constant__ RuleConfig rule, double alpha, const double *norm2,
+                       double *uhist, bool filled, float *weights, int nworkers)
 {
     const int i = threadIdx.x;
     if (i < nworkers) {
         double *ring = uhist + (size_t)i * (rule.p_hist + 1);
-        weight_rule_step(rule, norm2[i], ring, ring, filled, &weights[i], &weights[nworkers + i]);
+        weight_rule_step(rule.p_hist, rule.coef, rule.kappa, alpha, norm2[i], ring, ring, filled,
+                         &weights[i], &weights[nworkers + i]);
     }
 }
 
@@ -32,12 +35,12 @@ int ah::enqueue_weight_rule(ah_ctx *h, float alpha)
     const int rc = ring_to_device(h);
     if (rc != AH_OK) return rc;
     const bool filled = h->ring_home == 1 || h->ring_filled != 0;
-    WeightRule rule;
+    RuleConfig rule;
+    memset(&rule, 0, sizeof rule);
     rule.p_hist = h->p_hist;
-    for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = j < h->p_hist ? h->coef[j] : 0.0;
+    for (int j = 0; j < h->p_hist; ++j) rule.coef[j] = h->coef[j];
     rule.kappa = h->kappa;
-    rule.alpha = (double)alpha;
-    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, h->norm2_dev + 1,
+    dynamic_weights_kernel<<<1, AH_MAX_WORKERS, 0, h->stream>>>(rule, (double)alpha, h->norm2_dev + 1,
                                                                  h->ring_dev[h->ring_cur], filled,
                                                                  h->weights_dev, h->K);
     const cudaError_t e = cudaGetLastError();

@@ -60,6 +60,12 @@ uint32_t tree_shape(uint32_t ntiles, uint32_t ntp, uint32_t K, DistTree &T)
     T.levels = L;
     for (uint32_t q = L + 1; q <= (uint32_t)kTreeMaxLevels; ++q) T.n[q] = T.live[q] = T.off[q] = 0u;
     T.K = K;
+    // node / live[q] == mulhi(node, ceil(2^32 / live[q])) for every node < K * live[q] as long
+    // as K * live[q]^2 < 2^32; otherwise (magic 0) the kernels divide
+    for (uint32_t q = 0; q <= (uint32_t)kTreeMaxLevels; ++q) {
+        const uint64_t d = T.live[q];
+        T.magic[q] = d > 1u && (uint64_t)K * d * d < (1ull << 32) ? (uint32_t)(((1ull << 32) + d - 1) / d) : 0u;
+    }
     T.shared_levels = 0;
     for (uint32_t q = 1; q <= L; ++q)
         if ((uint64_t)K * T.live[q - 1] > kTreeOwnLevelInputs) T.shared_levels = q;
@@ -227,19 +233,19 @@ void ah::commit_distance_store(ah_ctx *h, bool rule, float alpha, bool owed_to_e
     if (owed_to_exchange) h->rule_fresh_alpha = alpha;
 }
 
-// A launch is about to assemble the waiting tile sums at its head (its first sync_ctas
-// CTAs share the large levels), and to run the weighting rule on the result if asked.
-int ah::begin_assembly(ah_ctx *h, bool run_rule, float alpha, uint32_t sync_ctas, DistTree &tree)
+// A launch is about to assemble the waiting tile sums at its head, and to run the
+// weighting rule on the result if asked.
+int ah::begin_assembly(ah_ctx *h, bool run_rule, float alpha, DistTree &tree)
 {
     if (h->tree_dirty) {          // an earlier kernel stopped half way
         AH_CUDA(h, cudaMemsetAsync(h->tree.arrive, 0, (kTreeMaxLevels + 1) * sizeof(uint32_t), h->stream));
-        h->arrive_total = 0;
+        memset(h->arrive_total, 0, sizeof h->arrive_total);
         h->tree_dirty = false;
     }
     tree.assemble = 1u;
     tree.sums_in = h->sums[h->sums_cur];
-    tree.sync_ctas = sync_ctas;
-    tree.arrive_target = h->arrive_total + sync_ctas;
+    for (uint32_t L = 1; L <= tree.shared_levels; ++L)     // the counters count finished nodes
+        tree.arrive_target[L] = h->arrive_total[L] + tree.K * tree.live[L];
     tree.wait_polls = h->wait_polls;
     tree.run_rule = run_rule ? 1u : 0u;
     tree.rule_alpha = (double)alpha;
@@ -262,7 +268,7 @@ int ah::begin_assembly(ah_ctx *h, bool run_rule, float alpha, uint32_t sync_ctas
 // wait for; the rule's bookkeeping follows.
 int ah::commit_assembly(ah_ctx *h, const DistTree &tree)
 {
-    h->arrive_total = tree.arrive_target;
+    for (uint32_t L = 1; L <= tree.shared_levels; ++L) h->arrive_total[L] = tree.arrive_target[L];
     h->sums_raw = false;
     if (tree.run_rule) {
         h->ring_cur ^= 1;
@@ -280,14 +286,14 @@ int ah::settle_distances(ah_ctx *h)
 {
     if (!h->has_device || !h->sums_raw) return AH_OK;
     DistTree tree = h->tree;
-    // one warp a node of the first level, four warps a CTA, at most one CTA per SM
+    // one warp a node of the first level, four warps a CTA, at most two CTAs per SM
     const uint64_t nodes = (uint64_t)h->K * tree.live[1];
     uint32_t ctas = (uint32_t)((nodes + 3) / 4);
-    if (ctas > (uint32_t)h->sm_count) ctas = (uint32_t)h->sm_count;
+    if (ctas > 2u * (uint32_t)h->sm_count) ctas = 2u * (uint32_t)h->sm_count;
     if (ctas < 1u) ctas = 1u;
-    const int rc = begin_assembly(h, h->raw_rule, h->raw_alpha, ctas, tree);
+    const int rc = begin_assembly(h, h->raw_rule, h->raw_alpha, tree);
     if (rc != AH_OK) return rc;
-    AH_CUDA(h, launch_assemble(tree, h->stream));
+    AH_CUDA(h, launch_assemble(tree, ctas, h->stream));
     h->launches += 1;
     return commit_assembly(h, tree);
 }
@@ -596,9 +602,7 @@ int local_step_impl(ah_ctx *h, const float *grad, const float *hvp, uint64_t ld,
     }
     p.tree = h->tree;
     if (assemble_here) {
-        // its first CTAs share the large levels: the grid has at least this many
-        const uint32_t sync_ctas = p.nitems < (uint32_t)h->sm_count ? p.nitems : (uint32_t)h->sm_count;
-        const int rc = begin_assembly(h, rule_at_head, head_alpha, sync_ctas, p.tree);
+        const int rc = begin_assembly(h, rule_at_head, head_alpha, p.tree);
         if (rc != AH_OK) return rc;
     }
     if (dist) {
@@ -818,16 +822,11 @@ int dw_weights_from_norm2(ah_ctx *h, const double *norm2, float alpha, float *we
     if (rc != AH_OK) return rc;
     memcpy(h->norm2_last, norm2, h->K * sizeof(double));
 
-    WeightRule rule;
-    rule.p_hist = h->p_hist;
-    memcpy(rule.coef, h->coef, sizeof(rule.coef));
-    rule.kappa = h->kappa;
-    rule.alpha = (double)alpha;
     const int depth = h->p_hist + 1;
     for (int i = 0; i < h->K; ++i) {
         double *ring = &h->uhist[(size_t)i * depth];
-        weight_rule_step(rule, h->norm2_last[i], ring, ring, h->ring_filled != 0, &weights[i],
-                         &weights[h->K + i]);
+        weight_rule_step(h->p_hist, h->coef, h->kappa, (double)alpha, h->norm2_last[i], ring, ring,
+                         h->ring_filled != 0, &weights[i], &weights[h->K + i]);
     }
     h->ring_filled = 1;
     return AH_OK;

@@ -103,15 +103,15 @@ struct RuleConfig {
 // every higher level holds, per worker, the adjacent-pairs tree sums of 64 consecutive
 // nodes of the level below, up to a single root, norm2[i].  The upper levels are formed at
 // the head of the launch that needs the distances (the fused exchange that follows, or a
-// small kernel of its own for every other reader): the first `sync_ctas` CTAs share the
-// nodes of the large levels and meet at one arrival counter per level; levels with few
+// small kernel of its own for every other reader): the CTAs share the nodes of the large
+// levels and meet at one counter per level, which counts finished nodes; levels with few
 // inputs are summed by every CTA for itself.  A CTA that has waited `wait_polls` polls for
 // the others sums the whole level itself, so nothing depends on the CTAs running at the
 // same time; the values are the same whoever forms them (fixed tree order).  CTA 0 also
 // copies the K results (and the status word) to pinned host memory and, when the rule is
 // asked for, stores the coefficients and the advanced history ring.  Level 0 has two
 // copies, so that a launch may assemble one round's sums while it stores the next one's.
-// The arrival counters only ever grow: a launch is told the value they reach with it.
+// The counters only ever grow: a launch is told the values they reach with it.
 constexpr int kTreeRadixLog2 = 6;
 constexpr int kTreeMaxLevels = 4;      // 2^21 tiles at most (P < 2^31, 1024 parameters a tile)
 constexpr uint32_t kTreeOwnLevelInputs = 1024;   // a level with at most this many inputs (all
@@ -121,7 +121,7 @@ struct DistTree {
                                        //   rounded up to a power of two
     const double *sums_in;             // level 0 this launch assembles (assemble != 0)
     double *upper;                     // level L >= 1: upper + K * off[L] + i * n[L] + node
-    uint32_t *arrive;                  // [L]: CTAs that have delivered their share of level L
+    uint32_t *arrive;                  // [L]: nodes of level L finished so far, over all launches
     double *norm2;                     // [K] roots
     double *norm2_host;                // pinned, mapped: [0] status word, [1 .. K] roots
     const uint32_t *status;            // device status word
@@ -133,8 +133,8 @@ struct DistTree {
     uint32_t ring_filled;              // 0: the ring holds no sample yet
     uint32_t run_rule;                 // 1: run the rule on the assembled distances
     uint32_t assemble;                 // 1: this launch assembles sums_in at its head
-    uint32_t sync_ctas;                // CTAs 0 .. sync_ctas-1 share the large levels
-    uint32_t arrive_target;            // what arrive[L] reaches when they all have delivered
+    uint32_t arrive_target[kTreeMaxLevels + 1];   // what arrive[L] reaches when this launch's
+                                       //   nodes of level L are all finished
     uint32_t wait_polls;               // polls before a CTA stops waiting for the others
     uint32_t shared_levels;            // levels 1 .. shared_levels are the large ones
     uint32_t K;
@@ -142,6 +142,7 @@ struct DistTree {
     uint32_t n[kTreeMaxLevels + 1];    // nodes per worker at each level
     uint32_t live[kTreeMaxLevels + 1]; // of which exist (the others count as +0, never read)
     uint32_t off[kTreeMaxLevels + 1];  // nodes per worker in the levels 1 .. L-1
+    uint32_t magic[kTreeMaxLevels + 1];// ceil(2^32 / live[L]) where node / live[L] is that mul-hi, else 0
 };
 
 // Launch parameters of the fused local step.  The per-worker tables are sized by the

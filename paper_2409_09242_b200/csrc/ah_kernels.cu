@@ -85,22 +85,22 @@ broadcast_kernel(float *x, const float *c, uint64_t lds, uint32_t nvec)
 
 // The distances ||x_i - c||^2 from the tile sums of the last distance round (and the
 // weighting rule on them, if it is owed), for the host, a snapshot or an exchange kernel:
-// T.sync_ctas CTAs of four warps.
+// a few CTAs of four warps.
 constexpr int kAssembleThreads = 128;
 __global__ void __launch_bounds__(kAssembleThreads)
 assemble_kernel(const __grid_constant__ DistTree T)
 {
-    __shared__ uint32_t word;
-    assemble_distances(T, (int)threadIdx.x, kAssembleThreads, blockIdx.x, nullptr, nullptr, &word,
-                       [] { __syncthreads(); });
+    __shared__ uint32_t words[2];
+    assemble_distances(T, (int)threadIdx.x, kAssembleThreads, blockIdx.x, gridDim.x, nullptr, nullptr,
+                       words, [] { __syncthreads(); }, [] {});
 }
 
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-cudaError_t launch_assemble(const DistTree &T, cudaStream_t s)
+cudaError_t launch_assemble(const DistTree &T, uint32_t ctas, cudaStream_t s)
 {
-    assemble_kernel<<<T.sync_ctas, kAssembleThreads, 0, s>>>(T);
+    assemble_kernel<<<ctas, kAssembleThreads, 0, s>>>(T);
     return cudaGetLastError();
 }
 

@@ -87,32 +87,43 @@ __host__ __device__ inline Pair pair_reciprocal(double n)
 
 // The same pairs for the odd n = 3, 5, ..., 43 of the series, written out (entry k holds
 // 1 / (2k + 3)), so that the series costs no divisions; a host test recomputes them with
-// pair_reciprocal.
+// pair_reciprocal.  Kept as a table (constant memory on the device) so that the series
+// can be a loop: the rule runs once per launch, where short code starts faster.
+#define AH_SERIES_RECIPROCALS {                                              \
+    {0x1.5555555555555p-2, 0x1.5555555555555p-56}  /* 1 / 3 */, \
+    {0x1.999999999999ap-3, -0x1.999999999999ap-57}  /* 1 / 5 */, \
+    {0x1.2492492492492p-3, 0x1.2492492492492p-57}  /* 1 / 7 */, \
+    {0x1.c71c71c71c71cp-4, 0x1.c71c71c71c71cp-58}  /* 1 / 9 */, \
+    {0x1.745d1745d1746p-4, -0x1.745d1745d1746p-59}  /* 1 / 11 */, \
+    {0x1.3b13b13b13b14p-4, -0x1.3b13b13b13b14p-58}  /* 1 / 13 */, \
+    {0x1.1111111111111p-4, 0x1.1111111111111p-60}  /* 1 / 15 */, \
+    {0x1.e1e1e1e1e1e1ep-5, 0x1.e1e1e1e1e1e1ep-61}  /* 1 / 17 */, \
+    {0x1.af286bca1af28p-5, 0x1.af286bca1af28p-59}  /* 1 / 19 */, \
+    {0x1.8618618618618p-5, 0x1.8618618618618p-59}  /* 1 / 21 */, \
+    {0x1.642c8590b2164p-5, 0x1.642c8590b2164p-60}  /* 1 / 23 */, \
+    {0x1.47ae147ae147bp-5, -0x1.eb851eb851eb8p-61}  /* 1 / 25 */, \
+    {0x1.2f684bda12f68p-5, 0x1.2f684bda12f68p-59}  /* 1 / 27 */, \
+    {0x1.1a7b9611a7b96p-5, 0x1.1a7b9611a7b96p-61}  /* 1 / 29 */, \
+    {0x1.0842108421084p-5, 0x1.0842108421084p-60}  /* 1 / 31 */, \
+    {0x1.f07c1f07c1f08p-6, -0x1.f07c1f07c1f08p-61}  /* 1 / 33 */, \
+    {0x1.d41d41d41d41dp-6, 0x1.0750750750750p-60}  /* 1 / 35 */, \
+    {0x1.bacf914c1bad0p-6, -0x1.bacf914c1bad0p-60}  /* 1 / 37 */, \
+    {0x1.a41a41a41a41ap-6, 0x1.0690690690690p-60}  /* 1 / 39 */, \
+    {0x1.8f9c18f9c18fap-6, -0x1.f3831f3831f38p-61}  /* 1 / 41 */, \
+    {0x1.7d05f417d05f4p-6, 0x1.7d05f417d05f4p-62}  /* 1 / 43 */ }
+static const double kSeriesReciprocalHost[21][2] = AH_SERIES_RECIPROCALS;
+#ifdef __CUDACC__
+static __constant__ double kSeriesReciprocalDevice[21][2] = AH_SERIES_RECIPROCALS;
+#endif
+#undef AH_SERIES_RECIPROCALS
+
 __host__ __device__ inline Pair series_reciprocal(int k)
 {
-    switch (k) {
-    case 0: return Pair{0x1.5555555555555p-2, 0x1.5555555555555p-56};     // 1 / 3
-    case 1: return Pair{0x1.999999999999ap-3, -0x1.999999999999ap-57};     // 1 / 5
-    case 2: return Pair{0x1.2492492492492p-3, 0x1.2492492492492p-57};     // 1 / 7
-    case 3: return Pair{0x1.c71c71c71c71cp-4, 0x1.c71c71c71c71cp-58};     // 1 / 9
-    case 4: return Pair{0x1.745d1745d1746p-4, -0x1.745d1745d1746p-59};     // 1 / 11
-    case 5: return Pair{0x1.3b13b13b13b14p-4, -0x1.3b13b13b13b14p-58};     // 1 / 13
-    case 6: return Pair{0x1.1111111111111p-4, 0x1.1111111111111p-60};     // 1 / 15
-    case 7: return Pair{0x1.e1e1e1e1e1e1ep-5, 0x1.e1e1e1e1e1e1ep-61};     // 1 / 17
-    case 8: return Pair{0x1.af286bca1af28p-5, 0x1.af286bca1af28p-59};     // 1 / 19
-    case 9: return Pair{0x1.8618618618618p-5, 0x1.8618618618618p-59};     // 1 / 21
-    case 10: return Pair{0x1.642c8590b2164p-5, 0x1.642c8590b2164p-60};     // 1 / 23
-    case 11: return Pair{0x1.47ae147ae147bp-5, -0x1.eb851eb851eb8p-61};     // 1 / 25
-    case 12: return Pair{0x1.2f684bda12f68p-5, 0x1.2f684bda12f68p-59};     // 1 / 27
-    case 13: return Pair{0x1.1a7b9611a7b96p-5, 0x1.1a7b9611a7b96p-61};     // 1 / 29
-    case 14: return Pair{0x1.0842108421084p-5, 0x1.0842108421084p-60};     // 1 / 31
-    case 15: return Pair{0x1.f07c1f07c1f08p-6, -0x1.f07c1f07c1f08p-61};     // 1 / 33
-    case 16: return Pair{0x1.d41d41d41d41dp-6, 0x1.0750750750750p-60};     // 1 / 35
-    case 17: return Pair{0x1.bacf914c1bad0p-6, -0x1.bacf914c1bad0p-60};     // 1 / 37
-    case 18: return Pair{0x1.a41a41a41a41ap-6, 0x1.0690690690690p-60};     // 1 / 39
-    case 19: return Pair{0x1.8f9c18f9c18fap-6, -0x1.f3831f3831f38p-61};     // 1 / 41
-    default: return Pair{0x1.7d05f417d05f4p-6, 0x1.7d05f417d05f4p-62};     // 1 / 43
-    }
+#ifdef __CUDA_ARCH__
+    return Pair{kSeriesReciprocalDevice[k][0], kSeriesReciprocalDevice[k][1]};
+#else
+    return Pair{kSeriesReciprocalHost[k][0], kSeriesReciprocalHost[k][1]};
+#endif
 }
 
 // ln x for a positive, finite, normal x.
@@ -146,7 +157,7 @@ __host__ __device__ inline double ln_pairwise(double x)
 
     const Pair z = pair_mul(s, s);
     Pair series = series_reciprocal(20);                       // 1 / 43
-#pragma unroll
+#pragma unroll 1
     for (int k = 20; k >= 1; --k)
         series = pair_add(pair_mul(series, z), series_reciprocal(k - 1));   // 1 / (2k + 1)
     const Pair unity = {1.0, 0.0};

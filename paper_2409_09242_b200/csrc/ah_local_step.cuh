@@ -307,7 +307,7 @@ struct __align__(128) Shared {
     uint64_t empty[kStages];               // consumers -> producer (stage drained)
     float h1[FUSE ? MAXW : 1];             // fused exchange: coefficients by worker index
     float h2[FUSE ? MAXW : 1];
-    uint32_t word;                         // fused exchange: scratch of the distance assembly
+    uint32_t words[2];                     // fused exchange: scratch of the distance assembly
 };
 
 // All consumers learn whether every one of them saw the stage arrive.
@@ -479,6 +479,12 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
         // round trip of the atomic overlaps the wait for a free stage.
         uint32_t drawn = 0;
         if (lane == 0) drawn = atomicAdd(&p.sched[0], 1u);
+        if constexpr (FUSE) {
+            // a launch that assembles distances at its head: the bulk copies start when the
+            // consumers have the tree's few small loads behind them (these would otherwise
+            // queue behind megabytes of tiles), and land while the rule is computed
+            if (p.tree.assemble) asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
+        }
         uint32_t k = 0;
         uint32_t tile = 0, r = 0, rows_left = 0;   // FUSE: where the producer is in a tile's worker list
         bool healthy = true;
@@ -613,8 +619,9 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
         // distances this launch assembles first, or from device memory, or from the launch
         const bool rule_here = p.tree.assemble != 0u && p.tree.run_rule != 0u;
         if (p.tree.assemble)
-            assemble_distances(p.tree, ctid, kConsumers, blockIdx.x, rule_here ? sh.h1 : nullptr,
-                               sh.h2, &sh.word, [] { consumer_sync(); });
+            assemble_distances(p.tree, ctid, kConsumers, blockIdx.x, gridDim.x,
+                               rule_here ? sh.h1 : nullptr, sh.h2, sh.words, [] { consumer_sync(); },
+                               [] { asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory"); });
         if (!rule_here)
             for (uint32_t w = (uint32_t)ctid; w < p.nworkers; w += (uint32_t)kConsumers) {
                 sh.h1[w] = p.wdev ? p.wdev[p.nworkers + w] : p.h1w[w];

@@ -19,6 +19,14 @@ __device__ __forceinline__ void fence_gpu()
     asm volatile("fence.acq_rel.gpu;" ::: "memory");
 }
 
+// node / per: one mul-hi where the host found that exact for every node of the level
+// (magic != 0), nothing at all at the root level.
+__device__ __forceinline__ uint32_t tree_worker_of(uint32_t node, uint32_t per, uint32_t magic)
+{
+    if (per == 1u) return node;
+    return magic ? __umulhi(node, magic) : node / per;
+}
+
 __device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t *p)
 {
     uint32_t v;
@@ -26,29 +34,38 @@ __device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t *p)
     return v;
 }
 
-// A distance round's only contribution: the tile's sum goes to its level-0 slot.
+// A distance round's only contribution: the tile's sum goes to its level-0 slot.  The line
+// is asked to stay in the L2 cache: it is read once more, at the head of a later launch,
+// after gigabytes of state have streamed past.
 __device__ __forceinline__ void tree_store_tile(const DistTree &T, uint32_t i, uint32_t tile, double v)
 {
-    T.sums_out[(size_t)i * T.n[0] + tile] = v;
+    uint64_t keep;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+    asm volatile("st.global.L2::cache_hint.f64 [%0], %1, %2;"
+                 :: "l"(T.sums_out + (size_t)i * T.n[0] + tile), "d"(v), "l"(keep) : "memory");
 }
 
 // Nodes first, first + stride, ... of level L (numbered worker by worker over the live
 // nodes), each by one warp: two children a lane, then the butterfly (the adjacent-pairs
-// order).  Four nodes' loads are in flight before the first sum is formed.
-__device__ __forceinline__ void tree_sum_nodes(const DistTree &T, uint32_t L, uint32_t first,
-                                               uint32_t stride, int lane)
+// order).  Four nodes' loads are in flight before the first sum is formed.  Returns how
+// many nodes this warp summed.  Out of line and short: one copy of the code serves every
+// level, and it runs once per launch, where fetching the instructions is most of the time.
+static __device__ __noinline__ uint32_t tree_sum_nodes(const DistTree &T, uint32_t L, uint32_t first,
+                                                       uint32_t stride, int lane)
 {
-    const uint32_t per = T.live[L], total = T.K * per;
+    constexpr int kBatch = 4;
+    const uint32_t per = T.live[L], total = T.K * per, magic = T.magic[L];
     const double *below = L == 1u ? T.sums_in : T.upper + (size_t)T.K * T.off[L - 1u];
     const uint32_t below_n = T.n[L - 1u], below_live = T.live[L - 1u];
-    for (uint32_t base = first; base < total; base += 4u * stride) {
-        double pair[4];
+    uint32_t done = 0;
+    for (uint32_t base = first; base < total; base += (uint32_t)kBatch * stride) {
+        double pair[kBatch];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kBatch; ++q) {
             const uint32_t node = base + (uint32_t)q * stride;
             pair[q] = 0.0;
             if (node < total) {
-                const uint32_t i = node / per, nd = node - i * per;
+                const uint32_t i = tree_worker_of(node, per, magic), nd = node - i * per;
                 const uint32_t children = min(1u << kTreeRadixLog2, below_live - (nd << kTreeRadixLog2));
                 const double *child = below + (size_t)i * below_n + ((size_t)nd << kTreeRadixLog2);
                 const uint32_t a = 2u * (uint32_t)lane, b = a + 1u;
@@ -58,32 +75,46 @@ __device__ __forceinline__ void tree_sum_nodes(const DistTree &T, uint32_t L, ui
             }
         }
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kBatch; ++q) {
             const uint32_t node = base + (uint32_t)q * stride;
             if (node < total) {                            // the same for every lane
                 const double sum = warp_tree_sum(pair[q]);
                 if (lane == 0) {
-                    const uint32_t i = node / per, nd = node - i * per;
+                    const uint32_t i = tree_worker_of(node, per, magic), nd = node - i * per;
                     if (L == T.levels) T.norm2[i] = sum;
                     else T.upper[(size_t)T.K * T.off[L] + (size_t)i * T.n[L] + nd] = sum;
                 }
+                ++done;
             }
         }
     }
+    return done;
 }
 
-// The whole assembly, by `nthreads` threads (whole warps) of every CTA of the launch;
-// `sync` is a barrier over exactly those threads and `scratch` one word of shared memory.
-// Afterwards every calling CTA may read norm2[0 .. K) (with __ldcg), and, if the rule was
-// asked for, finds the coefficients of worker w in h1s[w], h2s[w] (shared memory, may be
-// null).  Kept out of line: it runs once per launch, and its double-double logarithm
-// would otherwise claim registers in the streaming kernels.
-template <class Sync>
+// The whole assembly, by `nthreads` threads (whole warps) of every CTA of the launch (cta
+// of nctas); `sync` is a barrier over exactly those threads and `scratch` two words of
+// shared memory.  Afterwards every calling CTA may read norm2[0 .. K) (with __ldcg), and,
+// if the rule was asked for, finds the coefficients of worker w in h1s[w], h2s[w] (shared
+// memory; null where the caller does not use them).  `tree_done` is called by every thread
+// when the loads of the tree and of the rule are over: the moment for the caller's bulk
+// traffic to start, since those few small loads would otherwise queue behind it.  Kept out of
+// line: it runs once per launch, and its double-double logarithm would otherwise claim
+// registers in the streaming kernels.
+template <class Sync, class TreeDone>
 static __device__ __noinline__ void assemble_distances(const DistTree &T, int tid, int nthreads,
-                                                       uint32_t cta, float *h1s, float *h2s,
-                                                       uint32_t *scratch, Sync sync)
+                                                       uint32_t cta, uint32_t nctas, float *h1s,
+                                                       float *h2s, uint32_t *scratch, Sync sync,
+                                                       TreeDone tree_done)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
+    const size_t depth = (size_t)T.rule.p_hist + 1u;
+    if (T.run_rule && T.ring_filled)                       // the rule's history: on its way while
+        for (uint32_t w = (uint32_t)tid; w < T.K; w += (uint32_t)nthreads) {      // the sums form
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(T.ring_in + (size_t)w * depth));
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(T.ring_in + (size_t)w * depth + depth - 1u));
+        }
+    if (tid == 0) scratch[1] = 0u;
+    sync();
     for (uint32_t L = 1u; L <= T.levels; ++L) {
         if (L > T.shared_levels) {
             // few inputs: every CTA forms the whole level for itself (the CTAs store the
@@ -92,60 +123,61 @@ static __device__ __noinline__ void assemble_distances(const DistTree &T, int ti
             sync();
             continue;
         }
-        if (cta < T.sync_ctas)
-            tree_sum_nodes(T, L, cta * (uint32_t)nwarps + (uint32_t)warp,
-                           T.sync_ctas * (uint32_t)nwarps, lane);
-        sync();                                            // this CTA's share is stored
+        // this CTA's share of the level, then the count of what it finished
+        const uint32_t mine = tree_sum_nodes(T, L, cta * (uint32_t)nwarps + (uint32_t)warp,
+                                             nctas * (uint32_t)nwarps, lane);
+        if (lane == 0 && mine) atomicAdd(&scratch[1], mine);
+        sync();                                            // the share is stored and tallied
         if (tid == 0) {
-            if (cta < T.sync_ctas) {
-                fence_gpu();                               // ... and visible before it is counted
-                atomicAdd(&T.arrive[L], 1u);
+            const uint32_t finished = scratch[1];
+            scratch[1] = 0u;
+            if (finished) {
+                fence_gpu();                               // the sums are visible before they count
+                atomicAdd(&T.arrive[L], finished);
             }
             uint32_t polls = 0;
             bool there;
-            while (!(there = (int32_t)(ld_relaxed_gpu(&T.arrive[L]) - T.arrive_target) >= 0) &&
+            while (!(there = (int32_t)(ld_relaxed_gpu(&T.arrive[L]) - T.arrive_target[L]) >= 0) &&
                    polls < T.wait_polls) {
                 ++polls;
-                __nanosleep(64);
+                __nanosleep(32);
             }
             fence_gpu();                                   // what the counter announced is visible
-            *scratch = there ? 0u : 1u;
+            scratch[0] = there ? 0u : 1u;
         }
         sync();
-        const bool alone = *scratch != 0u;
-        sync();                                            // the word may be written again
-        if (alone) {                                       // the others are late: the whole level here
+        if (scratch[0] != 0u) {                            // the others are late: the whole level here
             tree_sum_nodes(T, L, (uint32_t)warp, (uint32_t)nwarps, lane);
             sync();
         }
     }
-    // ---- results to the host copy, the rule
-    WeightRule rule;
-    const size_t depth = (size_t)T.rule.p_hist + 1u;
-    if (T.run_rule) {
-        rule.p_hist = T.rule.p_hist;
-        for (int j = 0; j < AH_MAX_HIST; ++j) rule.coef[j] = T.rule.coef[j];
-        rule.kappa = T.rule.kappa;
-        rule.alpha = T.rule_alpha;
-    }
-    for (uint32_t w = (uint32_t)tid; w < T.K; w += (uint32_t)nthreads) {
-        const double n2 = __ldcg(&T.norm2[w]);
-        if (cta == 0u) T.norm2_host[1u + w] = n2;
-        if (T.run_rule) {
+    // ---- the rule, in every CTA of a launch that uses the coefficients (all of them finish
+    // it at the same moment: from here on nothing but arithmetic separates them from their
+    // first tile, and a CTA that fell behind would have to fetch through the others' traffic);
+    // CTA 0 stores what the rule leaves behind
+    const bool use_here = h1s != nullptr;
+    if (T.run_rule && (use_here || cta == 0u))
+        for (uint32_t w = (uint32_t)tid; w < T.K; w += (uint32_t)nthreads) {
+            const double n2 = __ldcg(&T.norm2[w]);
             float to_master, to_worker;
-            weight_rule_step(rule, n2, T.ring_in + (size_t)w * depth,
+            weight_rule_step(T.rule.p_hist, T.rule.coef, T.rule.kappa, T.rule_alpha, n2,
+                             T.ring_in + (size_t)w * depth,
                              cta == 0u ? T.ring_out + (size_t)w * depth : nullptr,
                              T.ring_filled != 0u, &to_master, &to_worker);
-            if (h1s) { h1s[w] = to_worker; h2s[w] = to_master; }
+            if (use_here) { h1s[w] = to_worker; h2s[w] = to_master; }
             if (cta == 0u) { T.weights[w] = to_master; T.weights[T.K + w] = to_worker; }
         }
-    }
-    if (cta == 0u && tid == 0) {
-        // the status word travels as the bit pattern of the first double, as it sits in
-        // device memory in front of the distances; the host reads its copy only behind an
-        // event that follows this kernel
-        reinterpret_cast<uint32_t *>(T.norm2_host)[0] = __ldcg(T.status);
-        reinterpret_cast<uint32_t *>(T.norm2_host)[1] = 0u;
+    tree_done();
+    if (cta == 0u) {
+        // results and status word to the host copy; the word travels as the bit pattern of
+        // the first double, as it sits in device memory in front of the distances; the host
+        // reads its copy only behind an event that follows this kernel
+        for (uint32_t w = (uint32_t)tid; w < T.K; w += (uint32_t)nthreads)
+            T.norm2_host[1u + w] = __ldcg(&T.norm2[w]);
+        if (tid == 0) {
+            reinterpret_cast<uint32_t *>(T.norm2_host)[0] = __ldcg(T.status);
+            reinterpret_cast<uint32_t *>(T.norm2_host)[1] = 0u;
+        }
     }
     sync();
 }
