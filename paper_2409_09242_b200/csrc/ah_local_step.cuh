@@ -447,14 +447,15 @@ __device__ __forceinline__ double stage_sum(const Stage<HASC> &st, int lane)
 // CTAs per SM an instantiation is built (register bound) and launched for.
 constexpr int ctas_per_sm(bool dist, bool multi, bool fuse)
 {
-    return dist || multi || fuse ? kCtasPerSm : kCtasPerSmPlain;
+    (void)dist;                 // a distance round's stages are those of a plain round
+    return multi || fuse ? kCtasPerSm : kCtasPerSmPlain;
 }
 
 template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE, int MAXW>
 __global__ void __launch_bounds__(kThreads, ctas_per_sm(DIST, MULTI, FUSE))
 local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
 {
-    constexpr bool HASC = DIST || FUSE;            // the stages carry a tile of the master row
+    constexpr bool HASC = FUSE;                    // the stages carry a tile of the master row
     extern __shared__ __align__(128) unsigned char smem_raw[];
     using SharedT = Shared<HASC, FUSE, MAXW>;
     SharedT &sh = *reinterpret_cast<SharedT *>(smem_raw);
@@ -562,7 +563,7 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                 const uint32_t row_bytes = n4 * 4u, hv_bytes = (ea1 - ea0) * 4u;
                 const uint64_t so = (uint64_t)i * p.lds + t0;
                 uint64_t *bar = &sh.full[s];
-                const bool want_c = FUSE ? first : DIST;      // fused: once per tile
+                const bool want_c = FUSE && first;            // fused: the master tile, once per tile
                 if (act) {
                     mbar_arrive_expect_tx(bar, 4u * row_bytes + (1u + nextra) * hv_bytes +
                                                    (want_c ? row_bytes : 0u));
@@ -578,10 +579,10 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                     bulk_load(st.m, p.m + so, row_bytes, bar);
                     bulk_load(st.v, p.v + so, row_bytes, bar);
                     if constexpr (HASC) if (want_c) bulk_load(st.c, p.c + t0, row_bytes, bar);
-                } else if constexpr (HASC) {
+                } else if constexpr (DIST || FUSE) {
                     mbar_arrive_expect_tx(bar, (want_c ? 2u : 1u) * row_bytes);
                     bulk_load(st.x, p.x + so, row_bytes, bar);
-                    if (want_c) bulk_load(st.c, p.c + t0, row_bytes, bar);
+                    if constexpr (HASC) if (want_c) bulk_load(st.c, p.c + t0, row_bytes, bar);
                 }
             }
             if constexpr (FUSE) { ++r; --rows_left; }
@@ -643,6 +644,17 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
         const ExtraSample *xs = extra + s * nextra;
         const float fn = (float)p.nsamp, rn = __frcp_rn(fn);
         float4 xn[kPasses];
+        // distance rounds without an exchange: the master values of this thread's columns come
+        // straight from memory (the L2 cache serves all workers of a tile but the first); asked
+        // for now, used after the step
+        float4 c_now[kPasses];
+        if constexpr (DIST && !FUSE) {
+#pragma unroll
+            for (int pass = 0; pass < kPasses; ++pass) {
+                const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
+                if (off < nvalid) c_now[pass] = ld_vec(p.c + t0 + off);
+            }
+        }
         // fused exchange: does this worker meet the master, with which coefficients, and
         // before its local step (the exchange of the previous round) or after it
         const bool meets = FUSE && (flags & kItemExchange) != 0u;
@@ -745,7 +757,7 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                     xn[pass] = x;
                 }
             }
-        } else if constexpr (HASC) {
+        } else if constexpr (DIST || FUSE) {
 #pragma unroll
             for (int pass = 0; pass < kPasses; ++pass) {
                 const uint32_t off = (uint32_t)pass * kPassElems + 4u * ctid;
@@ -767,7 +779,7 @@ local_step_kernel(const __grid_constant__ StepParamsT<MAXW> p)
                 double d = 0.0;
                 if (off < nvalid) {
                     const int nv = nvalid - off >= 4u ? 4 : (int)(nvalid - off);
-                    d = dist4(xn[pass], FUSE ? c_old[pass] : ld_vec(&st.c[off]), nv);
+                    d = dist4(xn[pass], FUSE ? c_old[pass] : c_now[pass], nv);
                 }
                 d = warp_tree_sum(d);
                 if (lane == 0) st.red[pass * kConsumerWarps + warp] = d;
@@ -810,7 +822,7 @@ template <int POWMODE, bool WD, bool DIST, bool MULTI, bool FUSE, int MAXW>
 static cudaError_t launch_step_one(const StepParamsT<MAXW> &p, int sm_count, cudaStream_t s)
 {
     auto kernel = local_step_kernel<POWMODE, WD, DIST, MULTI, FUSE, MAXW>;
-    constexpr bool HASC = DIST || FUSE;
+    constexpr bool HASC = FUSE;
     using SharedT = Shared<HASC, FUSE, MAXW>;
     const size_t smem = sizeof(SharedT) +
                         (MULTI ? (size_t)kStages * (p.nsamp - 1u) * sizeof(ExtraSample) : 0);
