@@ -173,7 +173,14 @@ __host__ __device__ inline double ln_pairwise(double x)
 
 // u = log ||x_i - c|| from the squared distance, clamped away from zero (workers
 // start as copies of the master, so the distance can be exactly 0).
-__host__ __device__ inline double u_from_norm2(double n2)
+// Out of line: one copy of the code per translation unit, so that on the device whoever
+// runs it first has fetched it for everybody after it.
+#ifdef __CUDACC__
+#define AH_NOINLINE __noinline__
+#else
+#define AH_NOINLINE __attribute__((noinline))
+#endif
+static __host__ __device__ AH_NOINLINE double u_from_norm2(double n2)
 {
     return AH_DMUL(0.5, ln_pairwise(n2 > 1e-300 ? n2 : 1e-300));
 }

@@ -115,6 +115,11 @@ static __device__ __noinline__ void assemble_distances(const DistTree &T, int ti
         }
     if (tid == 0) scratch[1] = 0u;
     sync();
+    // While the tree is formed (memory is quiet, and the last warp has the least to do), one
+    // thread runs the logarithm once for nothing: its instructions and constants are then at
+    // hand when the rule needs them, whatever the other CTAs are streaming by that time.
+    if (T.run_rule && h1s && warp == nwarps - 1 && lane == 31)
+        if (u_from_norm2(T.rule_alpha + 2.0) == -1.0) scratch[0] = 0u;      // never true
     for (uint32_t L = 1u; L <= T.levels; ++L) {
         if (L > T.shared_levels) {
             // few inputs: every CTA forms the whole level for itself (the CTAs store the
