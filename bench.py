@@ -58,8 +58,8 @@ HYPER = dict(lr=0.01, beta1=0.9, beta2=0.999, eps=1e-4, hessian_power=1.0, weigh
 # DRAM bytes per parameter update of the fused local-step kernel, from one ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch / (K * P)), and the hash
 # of the kernel sources it was taken on.  Reported only while the sources are unchanged.
-NCU_TRAFFIC = {"sources_sha256": "9ef6b32dec775a42983a3cdc8098b55fffb21311d610a211b12c1b79449e4ef2",
-               "dram_bytes_per_update": (935_959_040 + 506_229_504) / 46_758_048,
+NCU_TRAFFIC = {"sources_sha256": "21071469eb7f9ec7492ef6ad7b891cfb7db13d8c4eedcac99e44209bd09dbf6d",
+               "dram_bytes_per_update": (935_952_896 + 506_401_536) / 46_758_048,
                "capture": "one ncu capture of the plain local step on workload p18k4 (ResNet-18-shaped "
                           "layout, K=4, 46,758,048 updates per launch), scaled by the updates of this "
                           "run's launch: traffic is proportional to updates"}
@@ -67,7 +67,8 @@ NCU_TRAFFIC = {"sources_sha256": "9ef6b32dec775a42983a3cdc8098b55fffb21311d610a2
 
 def kernel_sources_hash() -> str:
     h = hashlib.sha256()
-    for fn in ("ah_local_step.cuh", "ah_step_inst.cu", "ah_tree.cuh", "ah_internal.h", "ah_device.cuh"):
+    for fn in ("ah_local_step.cuh", "ah_step_inst.cu", "ah_tree.cuh", "ah_weights.cuh", "ah_ln.cuh",
+               "ah_internal.h", "ah_device.cuh"):
         with open(os.path.join(ROOT, "paper_2409_09242_b200", "csrc", fn), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
