@@ -397,6 +397,57 @@ def test_riding_exchange_assembles_the_distances_without_a_launch_of_its_own(B, 
     assert np.all(seen[0][0] > 0)
 
 
+def test_a_rule_that_is_owed_runs_before_whatever_would_lose_it(B, torch):
+    # Tile sums wait until somebody needs the distances.  If the weighting rule is owed on them
+    # (AH_DIST_AND_RULE) and the next call would overwrite them (another distance round) or change
+    # the rule's setting (dw_config), the rule runs first: the history advances once per such
+    # round, exactly as when the host runs the rule after every distance round.
+    K, P = 3, 70_001
+    rng = np.random.default_rng(11)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    ld = W.padded_ld(P)
+    pairs = [(torch.from_numpy(rng.standard_normal((K, ld)).astype(np.float32)).cuda(),
+              torch.from_numpy(rng.standard_normal((K, ld)).astype(np.float32)).cuda()) for _ in range(3)]
+    mask = np.ones(K, np.uint8)
+    alpha = 0.07
+    c_new, kappa_new = np.array([0.5, 0.3, 0.2]), -0.2
+
+    def fresh():
+        h = B.Handle(K, P, [])
+        h.ah_state_set(B.AH_CENTER, theta0)
+        h.ah_broadcast_center()
+        return h
+
+    lazy, eager = fresh(), fresh()
+    # lazy: nobody looks at the distances between the rounds
+    for t in (1, 2, 3):
+        g, hv = pairs[t - 1]
+        lazy.ah_local_step(g, hv, 5, round_=t, lr=0.01, want_dist=B.AH_DIST_AND_RULE, rule_alpha=alpha)
+    lazy.dw_config(3, c_new, kappa_new)            # the rule owed on round 3 runs with the old setting
+    # eager: the host runs the rule after every distance round
+    for t in (1, 2, 3):
+        g, hv = pairs[t - 1]
+        eager.ah_local_step(g, hv, 5, round_=t, lr=0.01, want_dist=True)
+        w_eager = eager.dw_weights_next(alpha)
+    eager.dw_config(3, c_new, kappa_new)
+    assert np.array_equal(lazy.ah_state_get(B.AH_NORM2), eager.ah_state_get(B.AH_NORM2))
+    assert np.array_equal(lazy.ah_state_get(B.AH_UHIST, p_hist=3), eager.ah_state_get(B.AH_UHIST, p_hist=3))
+    assert np.array_equal(lazy.ah_state_get(B.AH_WEIGHTS), w_eager)
+    # one more period under the new setting, the exchange riding on the lazy side
+    g, hv = pairs[0]
+    lazy.ah_local_step(g, hv, 5, round_=4, lr=0.01, want_dist=B.AH_DIST_AND_RULE, rule_alpha=alpha)
+    lazy.easgd_exchange_then_step(g, hv, 5, round_=5, lr=0.01, worker_mask=mask, alpha=alpha, dynamic=True)
+    eager.ah_local_step(g, hv, 5, round_=4, lr=0.01, want_dist=True)
+    w = eager.dw_weights_next(alpha)
+    eager.easgd_exchange(mask, w, alpha)
+    eager.ah_local_step(g, hv, 5, round_=5, lr=0.01)
+    for which in (B.AH_X, B.AH_M, B.AH_V, B.AH_CENTER):
+        assert np.array_equal(lazy.ah_state_get(which), eager.ah_state_get(which)), which
+    assert np.array_equal(lazy.ah_state_get(B.AH_UHIST, p_hist=3), eager.ah_state_get(B.AH_UHIST, p_hist=3))
+    assert np.array_equal(lazy.ah_state_get(B.AH_WEIGHTS), w)
+    lazy.close(); eager.close()
+
+
 # --------------------------------------- weights on the device, no host round trip
 @pytest.mark.parametrize("asyn,mode", [(False, "yes"), (True, "yes"), (False, "mixed"), (True, "mixed")])
 def test_dynamic_exchange_on_device_matches_oracle(B, torch, asyn, mode):
